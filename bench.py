@@ -1,0 +1,390 @@
+#!/usr/bin/env python
+"""Benchmark of the SVD-Cache hot path on synthetic DiT-shaped feature streams.
+
+One "step" is one caching interval of the schedule over every block of the stream: one
+fused full step (project + residual + EMA, Eq. 8-11) followed by interval-1 fused cached
+steps (forecast + reconstruct, Sec. 3.5), each as ONE batched launch over all blocks.
+The metric is algorithmic HBM bytes per second over the whole step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload flux|hunyuan|dit_xl|tiny]
+    python bench.py --impl reference      # the fp64 CPU oracle on the host cores
+
+Under torchrun every rank runs its own copy of the stream (weak scaling, no data-path
+collective); rank 0 prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2601_07396_b200 import streams  # noqa: E402
+
+METRIC = "fused full/cached-step HBM GB/s and % of B200 HBM roofline (FLUX-shaped)"
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel (the
+# batched cached step), from the ncu capture summarised under profiles/ (captured on a
+# smaller block count and scaled by blocks, since traffic is proportional to blocks).
+# None until a capture exists for the workload.
+NCU_TRAFFIC_BYTES_PER_BLOCK = {}
+
+
+def algorithmic_bytes(spec: streams.StreamSpec, nblocks: int):
+    """Bytes the method must move per launch: F in / R out (full), R in / Fhat out
+    (cached), the fp32 coefficient arrays, and the basis once per block."""
+    N, D, k, b = spec.rows, spec.D, spec.k, spec.elem_bytes
+    full = 2 * N * D * b + 2 * N * k * 4 + 2 * D * k * b     # Chat read + write (C_out not requested); V and V^T
+    cached = 2 * N * D * b + N * k * 4 + D * k * b
+    return full * nblocks, cached * nblocks
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        inside = [r for (t, r) in self.rows if t0 <= t <= t1] or [r for (_, r) in self.rows[-3:]]
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in inside:
+            p = [x.strip() for x in r.split(",")]
+            try:
+                sm.append(float(p[0])); smax.append(float(p[1]))
+            except Exception:
+                continue
+            for nm, val in zip(names, p[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def reduce_max(value: float, world: int, device) -> float:
+    if world == 1:
+        return value
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+# ------------------------------------------------------------------------- ours ---
+
+def build_workload(spec, nblocks, device, block_offset=0, calibrate_rows=None):
+    """Features, calibrated bases and reset states for `nblocks` blocks, resident on the
+    device.  Returns dict of tensors."""
+    from paper_2601_07396_b200 import binding as sc
+    dt = sc.F32 if spec.dtype == "f32" else sc.BF16
+    N, D, k = spec.rows, spec.D, spec.k
+    F = torch.empty(nblocks, N, D, dtype=spec.torch_dtype, device=device)
+    bases = torch.empty(nblocks, sc.svdcache_basis_bytes(D, k, dt), dtype=torch.uint8, device=device)
+    ws = torch.empty(sc.svdcache_calibrate_workspace_bytes(D, k), dtype=torch.uint8, device=device)
+    cal_ms = []
+    n_cal = min(N, 4608) if calibrate_rows is None else calibrate_rows
+    for b in range(nblocks):
+        blk = block_offset + b
+        st = streams.BlockStream(spec, blk, trajectory=0, device=device)
+        st.features(0, out=F[b])
+        cal = streams.BlockStream(spec, blk, trajectory=1, device=device, rows=n_cal)
+        stack = cal.features(0)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        Vk, lam, tr, info = sc.svdcache_calibrate(stack, k, workspace=ws, strict=False)
+        e1.record()
+        torch.cuda.synchronize()
+        cal_ms.append(e0.elapsed_time(e1))
+        sc.svdcache_basis_prepare(Vk, dt, basis=bases[b])
+        del st, cal, stack
+    state = sc.new_state(N, D, k, dt, device, blocks=nblocks)
+    Fhat = torch.empty_like(F)
+    torch.cuda.synchronize()
+    return dict(F=F, bases=bases, state=state, Fhat=Fhat, dt=dt, cal_ms=cal_ms, cal_rows=n_cal)
+
+
+def run_ours(args):
+    from paper_2601_07396_b200 import binding as sc
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    sc.lib()
+
+    spec = streams.SPECS[args.workload]
+    nblocks = args.blocks or (spec.blocks if spec.name != "hunyuan" else 8)
+    wl = build_workload(spec, nblocks, device, block_offset=rank * spec.blocks)
+    F, bases, state, Fhat, dt = wl["F"], wl["bases"], wl["state"], wl["Fhat"], wl["dt"]
+    k, beta, interval = spec.k, spec.beta, spec.interval
+    bytes_full, bytes_cached = algorithmic_bytes(spec, nblocks)
+    step_bytes = bytes_full + (interval - 1) * bytes_cached
+
+    def one_step(events=None):
+        if events is not None:
+            e = torch.cuda.Event(enable_timing=True); e.record(); events.append(e)
+        sc.svdcache_full_step_batched(F, bases, state, k, beta)
+        if events is not None:
+            e = torch.cuda.Event(enable_timing=True); e.record(); events.append(e)
+        for j in range(1, interval):
+            sc.svdcache_cached_step_batched(state, bases, Fhat, k, steps_since_full=j)
+            if events is not None:
+                e = torch.cuda.Event(enable_timing=True); e.record(); events.append(e)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        one_step()
+    barrier()
+
+    # ---- device-resident timing: K steps, CUDA events on the launching stream ----
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.25)
+    launches0 = sc.svdcache_kernel_launches()
+    events = []
+    t_host0 = time.time()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(args.steps):
+        one_step(events)
+    stop.record()
+    barrier()
+    t_host1 = time.time()
+    clocks = sampler.stop(t_host0, t_host1)
+    launches = sc.svdcache_kernel_launches() - launches0
+    total_ms = reduce_max(start.elapsed_time(stop), world, device)
+    per = interval + 1
+    full_ms, cached_ms = [], []
+    for s in range(args.steps):
+        ev = events[s * per:(s + 1) * per]
+        full_ms.append(ev[0].elapsed_time(ev[1]))
+        for j in range(1, interval):
+            cached_ms.append(ev[j].elapsed_time(ev[j + 1]))
+    path_used = sc.svdcache_last_path()
+
+    # ---- end to end: host buffers, H2D of F and D2H of the final Fhat every step ----
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    F_host = torch.empty(F.shape, dtype=F.dtype, pin_memory=True)
+    F_host.copy_(F)
+    out_host = torch.empty(Fhat.shape, dtype=Fhat.dtype, pin_memory=True)
+    h2d = F_host.numel() * F_host.element_size()
+    d2h = out_host.numel() * out_host.element_size()
+    barrier()
+    s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s2.record()
+    for _ in range(e2e_steps):
+        F.copy_(F_host, non_blocking=True)
+        one_step()
+        out_host.copy_(Fhat, non_blocking=True)
+    e2.record()
+    barrier()
+    e2e_ms = reduce_max(s2.elapsed_time(e2), world, device)
+
+    if rank != 0:
+        return
+    peak, peak_kind = measured_peak()
+    value = world * step_bytes * args.steps / (total_ms * 1e-3) / 1e9
+    e2e_value = world * step_bytes * e2e_steps / (e2e_ms * 1e-3) / 1e9
+    cached_avg_ms = sum(cached_ms) / max(1, len(cached_ms))
+    full_avg_ms = sum(full_ms) / max(1, len(full_ms))
+    cached_gbs = bytes_cached / (cached_avg_ms * 1e-3) / 1e9 if cached_ms else None
+    full_gbs = bytes_full / (full_avg_ms * 1e-3) / 1e9
+    traffic = NCU_TRAFFIC_BYTES_PER_BLOCK.get((spec.name, path_used))
+    line = {
+        "metric": METRIC, "value": round(value, 2), "unit": "GB/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(total_ms / args.steps, 4),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if spec.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": f"{spec.name}-shaped stream", "blocks": nblocks, "rows": spec.rows,
+                   "D": spec.D, "k": spec.k, "interval": interval, "beta": beta,
+                   "step": f"1 batched full step + {interval - 1} batched cached steps over all blocks",
+                   "l2": "inputs larger than L2 (each launch streams >= 1 GB)" if step_bytes > 6e8 else
+                         "inputs smaller than L2: launch-bound parity config, not a roofline config",
+                   "kernel_family": {1: "cuda-core", 2: "tcgen05"}.get(path_used, "?"),
+                   "parallelism": f"blocks replicated per rank x{world}, no collective"},
+        "roofline": {"bound": "hbm", "kernel": "cached step (batched)",
+                     "achieved": round(cached_gbs, 2) if cached_gbs else None, "peak": peak,
+                     "peak_source": f"{peak_kind} copy bandwidth", "unit": "GB/s",
+                     "frac": round(cached_gbs / peak, 4) if cached_gbs else None,
+                     "frac_of_nominal_8TBs": round(cached_gbs / NOMINAL_HBM_GBS, 4) if cached_gbs else None,
+                     "traffic": traffic * nblocks if traffic else None,
+                     "algorithmic_bytes": bytes_cached, "avg_launch_ms": round(cached_avg_ms, 4)},
+        "roofline_full_step": {"bound": "hbm", "kernel": "full step (batched)", "achieved": round(full_gbs, 2),
+                               "peak": peak, "unit": "GB/s", "frac": round(full_gbs / peak, 4),
+                               "frac_of_nominal_8TBs": round(full_gbs / NOMINAL_HBM_GBS, 4),
+                               "algorithmic_bytes": bytes_full, "avg_launch_ms": round(full_avg_ms, 4)},
+        "tokens_blocks_per_s": round(world * spec.rows * nblocks * interval * args.steps / (total_ms * 1e-3), 1),
+        "e2e": {"value": round(e2e_value, 2), "unit": "GB/s", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                "note": "pinned host F copied in and final Fhat copied out every step"},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "calibration": {"rows": wl["cal_rows"], "median_ms_per_block": round(statistics.median(wl["cal_ms"]), 3),
+                        "note": "one-off per block, outside the timed steps"},
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(spec, F, bases, dt, budget_s=args.cpu_seconds)
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+# -------------------------------------------------------------- oracle-timed legs ---
+
+def _oracle_interval(oracle, Fh, V, beta, interval):
+    C, R, chat = oracle.full_step(Fh, V, beta, None)
+    for _ in range(interval - 1):
+        oracle.cached_step(chat, V, R)
+
+
+def cpu_baseline(spec, F, bases, dt, budget_s=12.0):
+    """The fp64 oracle as it stands, timed on this machine's host cores over whole blocks of
+    the same workload until `budget_s` seconds have been spent."""
+    from oracle import svdcache_oracle as oracle
+    from paper_2601_07396_b200 import binding as sc
+    import numpy as np
+    nb = F.shape[0]
+    rows = min(spec.rows, 2048)
+    done_bytes, t_spent, used = 0, 0.0, 0
+    sub = streams.StreamSpec(**{**spec.__dict__, "rows": rows})
+    bf, bc = algorithmic_bytes(sub, 1)
+    b = -1
+    while t_spent < budget_s:
+        b = (b + 1) % nb
+        V = (sc.basis_views(bases[b], spec.D, spec.k, dt)[0 if dt == sc.F32 else 2]).double().cpu().numpy()
+        Fh = F[b, :rows].double().cpu().numpy()
+        t0 = time.perf_counter()
+        _oracle_interval(oracle, Fh, V, float(np.float32(spec.beta)), spec.interval)
+        t_spent += time.perf_counter() - t0
+        done_bytes += bf + (spec.interval - 1) * bc
+        used += 1
+    return {"value": round(done_bytes / t_spent / 1e9, 4), "unit": "GB/s", "cores": oracle.threads(),
+            "kind": "oracle",
+            "sample": f"first {rows} rows of a block, {used} block passes: 1 full + {spec.interval - 1} cached steps each, "
+                      f"{t_spent:.1f} s of CPU work"}
+
+
+def run_reference(args):
+    """Reference arm: the fp64 CPU oracle on the host cores, on a bounded sample of the
+    same workload, metric and unit.  Rank 0 only."""
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    from oracle import svdcache_oracle as oracle
+    import numpy as np
+    spec = streams.SPECS[args.workload]
+    rows = min(spec.rows, args.ref_rows)
+    sub = streams.StreamSpec(**{**spec.__dict__, "rows": rows})
+    st = streams.BlockStream(spec, 0, device="cpu", rows=rows)
+    Fh = st.features(0).double().numpy()
+    V = st.V_gen[:, :spec.k].to(spec.torch_dtype).double().numpy()
+    bf, bc = algorithmic_bytes(sub, 1)
+    step_bytes = bf + (spec.interval - 1) * bc
+    beta = float(np.float32(spec.beta))
+    for _ in range(args.warmup):
+        _oracle_interval(oracle, Fh, V, beta, spec.interval)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        _oracle_interval(oracle, Fh, V, beta, spec.interval)
+    dt_s = time.perf_counter() - t0
+    value = step_bytes * args.steps / dt_s / 1e9
+    sample = f"{rows} rows of block 0 of the {spec.name}-shaped stream per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": round(value, 4), "unit": "GB/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dt_s * 1e3 / args.steps, 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{spec.name}-shaped stream", "rows": rows, "D": spec.D, "k": spec.k,
+                   "interval": spec.interval, "sample": sample},
+        "cpu_baseline": {"value": round(value, 4), "unit": "GB/s", "cores": oracle.threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": round(value, 4), "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="flux", choices=sorted(streams.SPECS))
+    ap.add_argument("--blocks", type=int, default=0, help="override the number of blocks")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--ref-rows", type=int, default=1024)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

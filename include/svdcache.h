@@ -1,0 +1,199 @@
+/*
+ * svdcache.h — C ABI of the B200-native SVD-Cache hot path (sm_100a).
+ *
+ * SVD-Cache ("Forecast the Principal, Stabilize the Residual") splits the hidden
+ * feature F (N tokens x D) of a DiT block into a rank-k principal part in a fixed,
+ * pre-computed right-singular basis V_k and an orthogonal residual, forecasts the
+ * principal part with an exponential moving average and reuses the residual:
+ *
+ *   one-off        V_k  = top-k right singular vectors of a stack of features  (Eq. 4-7)
+ *   full step      C    = F V_k                                                (Eq. 8-9)
+ *                  R    = F - C V_k^T                                          (Eq. 10)
+ *                  Chat = C  on the first full step, else beta Chat + (1-beta) C (Eq. 11)
+ *   cached step    Fhat = Chat V_k^T + R                                       (Sec. 3.5)
+ *
+ * Conventions
+ *   - Every function returns an int status: SVDCACHE_OK or a negative SVDCACHE_ERR_*.
+ *     Nothing throws.  svdcache_status_string() gives text.
+ *   - "device" pointers are CUDA device addresses owned by the caller; "host" pointers
+ *     are ordinary host addresses.  The library allocates no device memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  The step
+ *     and basis calls only enqueue work on it and return; they never synchronise.
+ *     Calls that must hand a number back to the host say so.
+ *   - Matrices are row-major.  `ld` is the row pitch in ELEMENTS (>= the row width).
+ *   - dtype is the storage type of F, R and Fhat: SVDCACHE_F32 or SVDCACHE_BF16.
+ *     Coefficients (C, Chat) are always fp32.  For SVDCACHE_BF16 the kernels read a
+ *     bf16 copy of V_k (made by svdcache_basis_prepare) and accumulate in fp32; for
+ *     SVDCACHE_F32 they read V_k in fp32 and accumulate in fp64.
+ *   - Shape limits: 1 <= N, 8 <= D <= 16384, D % 8 == 0, 8 <= k <= 256, k % 8 == 0,
+ *     k <= D.  F, R, Fhat, V_k and all library-defined buffers must be 16-byte aligned,
+ *     and (ld * element size) % 16 == 0.  Violations return SVDCACHE_ERR_BAD_SHAPE /
+ *     SVDCACHE_ERR_BAD_ALIGN before anything is launched.
+ *   - NaN / Inf in the inputs propagate per IEEE-754 and are not errors.
+ */
+#ifndef SVDCACHE_H_
+#define SVDCACHE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define SVDCACHE_API __attribute__((visibility("default")))
+#else
+#define SVDCACHE_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SVDCACHE_OK                0
+#define SVDCACHE_ERR_INVALID_ARG  (-1) /* NULL pointer, unknown dtype, bad scalar      */
+#define SVDCACHE_ERR_BAD_SHAPE    (-2) /* N, D, k, ld outside the limits above          */
+#define SVDCACHE_ERR_BAD_ALIGN    (-3) /* a pointer or pitch is not 16-byte aligned     */
+#define SVDCACHE_ERR_STATE        (-4) /* cached step on a state that saw no full step  */
+#define SVDCACHE_ERR_WORKSPACE    (-5) /* workspace / buffer smaller than required      */
+#define SVDCACHE_ERR_TIMEOUT      (-6) /* a bounded in-kernel wait ran out              */
+#define SVDCACHE_ERR_CUDA         (-7) /* a CUDA runtime / driver call failed           */
+#define SVDCACHE_ERR_NOT_CONVERGED (-8) /* eigen-solver hit its iteration limit         */
+
+#define SVDCACHE_F32   0
+#define SVDCACHE_BF16  1
+
+/* Text for a status code (static storage, never NULL). */
+SVDCACHE_API const char *svdcache_status_string(int status);
+
+/* Text of the last CUDA error seen by the calling thread inside this library. */
+SVDCACHE_API const char *svdcache_last_cuda_error(void);
+
+/* ---------------------------------------------------------------------------------
+ * Calibration: the "one-time SVD" of Sec. 3.3 (Eq. 4, Eq. 5, Eq. 7).
+ *
+ * The right singular vectors of a row-stack Fstack (M x D) are the eigenvectors of the
+ * Gram matrix G = Fstack^T Fstack, and sigma_i^2 its eigenvalues.  The stack may be fed
+ * in pieces: begin, accumulate (any number of times, any row counts), finish.
+ *
+ *   workspace  device, caller-owned scratch of at least
+ *              svdcache_calibrate_workspace_bytes(D, k) bytes, 256-byte aligned; it
+ *              carries G between the three calls and must not be touched in between.
+ *   F          device, M x D rows of dtype `dtype` with pitch ld; only read.
+ *   Vk         device, out: D x k fp32, orthonormal columns ordered by descending
+ *              eigenvalue; in each column the entry of largest magnitude is positive.
+ *   lambda     device, out, k doubles (eigenvalues of G = sigma_i^2), or NULL.
+ *   trace      device, out, 1 double: trace(G) = |Fstack|_F^2 = sum of ALL sigma_i^2
+ *              (the denominator of the energy criterion, Eq. 6), or NULL.
+ *   info       host, out, 4 doubles or NULL: {multiplications by G done, largest
+ *              relative eigen-residual |G v - lambda v| / lambda_1 over the k pairs,
+ *              Ritz block width, Jacobi sweeps of the last Rayleigh-Ritz step}.
+ *
+ * begin and accumulate only enqueue work.  finish synchronises `stream` several times
+ * (it reads convergence numbers back) and returns SVDCACHE_ERR_NOT_CONVERGED if the
+ * residual target was not met within the iteration limit (outputs are still written).
+ * G is accumulated in fp64 in a fixed order: results are bit-reproducible run to run.
+ * ------------------------------------------------------------------------------- */
+SVDCACHE_API int svdcache_calibrate_workspace_bytes(int D, int k, size_t *bytes /* host, out */);
+SVDCACHE_API int svdcache_calibrate_begin(int D, int k, void *workspace, size_t workspace_bytes, void *stream);
+SVDCACHE_API int svdcache_calibrate_accumulate(const void *F, int64_t M, int D, int64_t ld, int dtype,
+                                  void *workspace, size_t workspace_bytes, void *stream);
+SVDCACHE_API int svdcache_calibrate_finish(int D, int k, float *Vk, double *lambda, double *trace,
+                              double *info, void *workspace, size_t workspace_bytes,
+                              void *stream);
+/* One-shot form: begin + accumulate(Fstack) + finish. */
+SVDCACHE_API int svdcache_calibrate(const void *Fstack, int64_t M, int D, int64_t ld, int dtype, int k,
+                       float *Vk, double *lambda, double *trace, double *info,
+                       void *workspace, size_t workspace_bytes, void *stream);
+
+/* Rank selection by energy threshold (Eq. 6): the smallest k' <= n with
+ * sum_{i<=k'} lambda_i / trace >= tau; n if the n listed eigenvalues fall short.
+ * lambda: HOST array of n descending eigenvalues.  Pure host arithmetic. */
+SVDCACHE_API int svdcache_rank_for_energy(const double *lambda, int n, double trace, double tau,
+                             int *k_out /* host, out */);
+
+/* ---------------------------------------------------------------------------------
+ * Basis buffer: the cached reference basis of Eq. 7 in the layouts the step kernels
+ * read.  Layout (all sections 256-byte aligned, offsets from svdcache_basis_layout):
+ *   header (256 B) | V fp32 [D x k] | V^T fp32 [k x D] | V bf16 [D x k] | V^T bf16 [k x D]
+ * The two bf16 sections exist only for dtype = SVDCACHE_BF16; they hold V_k rounded to
+ * nearest-even, and are the values the bf16 kernels multiply with.
+ * ------------------------------------------------------------------------------- */
+SVDCACHE_API int svdcache_basis_bytes(int D, int k, int dtype, size_t *bytes /* host, out */);
+SVDCACHE_API int svdcache_basis_layout(int D, int k, int dtype,
+                          size_t *v_f32_offset, size_t *vt_f32_offset,
+                          size_t *v_bf16_offset, size_t *vt_bf16_offset /* host, out; may be NULL */);
+/* Vk: device D x k fp32 (only read).  basis: device, out, >= svdcache_basis_bytes. */
+SVDCACHE_API int svdcache_basis_prepare(const float *Vk, int D, int k, int dtype, void *basis,
+                           size_t basis_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------------
+ * Per-block cache state, a caller-owned flat device buffer (checkpoint = memcpy):
+ *   header (256 B) | Chat fp32 [N x k] | R dtype [N x D]          (dense, no pitch)
+ * The header counts the full steps the state has seen and carries a sticky device
+ * status word.  svdcache_state_reset must be called once before first use (and again to
+ * start a new sampling run): it clears the counter, so the next full step initialises
+ * the EMA with Chat = C.
+ * ------------------------------------------------------------------------------- */
+SVDCACHE_API int svdcache_state_bytes(int64_t N, int D, int k, int dtype, size_t *bytes /* host, out */);
+SVDCACHE_API int svdcache_state_layout(int64_t N, int D, int k, int dtype,
+                          size_t *chat_offset, size_t *r_offset /* host, out */);
+SVDCACHE_API int svdcache_state_reset(void *state, int64_t N, int D, int k, int dtype, void *stream);
+/* Synchronises `stream`, then reads the header: full steps seen, device status word
+ * (SVDCACHE_OK, SVDCACHE_ERR_STATE or SVDCACHE_ERR_TIMEOUT).  Outputs are host. */
+SVDCACHE_API int svdcache_state_query(const void *state, void *stream, int64_t *full_steps, int *status);
+
+/* ---------------------------------------------------------------------------------
+ * Full step (Eq. 8 - Eq. 11), one fused pass: C = F V_k, R = F - C V_k^T stored into
+ * the state, Chat updated in the state (Chat = C if the state has seen no full step
+ * yet).  F passes through untouched: the sampler keeps using the true feature.
+ *   F      device, N x D, pitch ld, only read
+ *   basis  device, from svdcache_basis_prepare for the same D, k, dtype
+ *   state  device, in/out
+ *   C_out  device, out, N x k fp32 (this step's coefficients), or NULL
+ *   beta   EMA weight in [0, 1] (the paper uses 0.9)
+ * ------------------------------------------------------------------------------- */
+SVDCACHE_API int svdcache_full_step(const void *F, int64_t ld, const void *basis, void *state,
+                       float *C_out, int64_t N, int D, int k, int dtype, float beta,
+                       void *stream);
+
+/* ---------------------------------------------------------------------------------
+ * Cached step (Sec. 3.5): Fhat = Chat V_k^T + R.  The EMA state changes only at full
+ * steps, so every cached step until the next full step returns the same Fhat;
+ * `steps_since_full` is accepted for predictors that extrapolate and is ignored by the
+ * EMA.  If the state has seen no full step the kernel writes nothing and records
+ * SVDCACHE_ERR_STATE in the state header (read it with svdcache_state_query).
+ *   Fhat   device, out, N x D, pitch ld
+ * ------------------------------------------------------------------------------- */
+SVDCACHE_API int svdcache_cached_step(const void *state, const void *basis, void *Fhat, int64_t ld,
+                         int64_t N, int D, int k, int dtype, int steps_since_full,
+                         void *stream);
+
+/* ---------------------------------------------------------------------------------
+ * Batched forms: the same operation on `nblocks` independent DiT blocks in ONE launch
+ * (Eq. 8 - Eq. 11 / Sec. 3.5 per block).  Block b uses F + b*F_stride, basis +
+ * b*basis_stride, state + b*state_stride, out + b*out_stride; all strides are in BYTES
+ * and multiples of 256.  Shapes, dtype and beta are shared.
+ * ------------------------------------------------------------------------------- */
+SVDCACHE_API int svdcache_full_step_batched(int nblocks, const void *F, int64_t ld, size_t F_stride,
+                               const void *basis, size_t basis_stride, void *state,
+                               size_t state_stride, float *C_out, size_t C_stride,
+                               int64_t N, int D, int k, int dtype, float beta, void *stream);
+SVDCACHE_API int svdcache_cached_step_batched(int nblocks, const void *state, size_t state_stride,
+                                 const void *basis, size_t basis_stride, void *Fhat,
+                                 int64_t ld, size_t Fhat_stride, int64_t N, int D, int k,
+                                 int dtype, int steps_since_full, void *stream);
+
+/* ---------------------------------------------------------------------------------
+ * Introspection for benchmarks and tests (host only).
+ *   svdcache_kernel_launches: kernels this library has launched in this process.
+ *   svdcache_set_path: 0 = pick automatically, 1 = force the CUDA-core kernels,
+ *                      2 = force the tcgen05 kernels (error if the shape is outside
+ *                      what they support).  Returns the previous setting.
+ *   svdcache_last_path: which kernel family the last step call used (1 or 2).
+ * ------------------------------------------------------------------------------- */
+SVDCACHE_API uint64_t svdcache_kernel_launches(void);
+SVDCACHE_API int svdcache_set_path(int path);
+SVDCACHE_API int svdcache_last_path(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SVDCACHE_H_ */

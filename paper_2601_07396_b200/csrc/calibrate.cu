@@ -1,0 +1,607 @@
+// Calibration path: the "one-time SVD" (Eq. 4, Eq. 5, Eq. 7) through the Gram matrix.
+//
+//   G = Fstack^T Fstack                accumulated in fp64 over any number of row chunks
+//   V_k = top-k eigenvectors of G      block subspace iteration with Rayleigh-Ritz:
+//        Z = G Q;  S = Q^T Z;  S = W Theta W^T (parallel cyclic Jacobi);  Q <- Q W;
+//        stop when |G v - theta v| <= tol * theta_1 for the k leading pairs;
+//        else Q <- orthonormalise(Z) (Cholesky-QR, applied twice) and repeat.
+//
+// Everything runs on the device in fp64 on the plain ALUs; the host only sequences
+// launches and reads one convergence number per Rayleigh-Ritz step.  The eigen-gap at k
+// of the power-law spectra met here is ~1e-6 of the leading eigenvalue, so fp32
+// anywhere in this path would miss a 1e-4 bound on the principal-angle cosines.
+#include <algorithm>
+#include <cmath>
+#include <utility>
+
+#include "internal.cuh"
+
+namespace svdc {
+
+bool umma_gram_supported(int64_t M, int D, int64_t ld, int dtype);
+int umma_gram_accumulate(const void *F, int64_t M, int D, int64_t ld, double *G, void *scratch,
+                         size_t scratch_bytes, cudaStream_t s);
+size_t umma_gram_scratch_bytes(int D);
+
+namespace {
+
+struct CalibHeader {
+    int32_t D, k_max;
+    int64_t rows;
+};
+
+int ritz_width(int D, int k) {
+    int p = std::max(16, k / 4);
+    int m = (k + p + 7) / 8 * 8;
+    return std::min(m, D);
+}
+
+struct CalibLayout {
+    size_t G, Q, Z, T, S, W, X, theta, resid, scal, dead, gram_scratch, total;
+    int m;
+};
+
+CalibLayout calib_layout(int D, int k) {
+    CalibLayout L;
+    L.m = ritz_width(D, k);
+    const size_t dm = align_up((size_t)D * L.m * 8, kAlign), mm = align_up((size_t)L.m * L.m * 8, kAlign);
+    size_t at = kHeaderBytes;
+    L.G = at; at += align_up((size_t)D * D * 8, kAlign);
+    L.Q = at; at += dm;
+    L.Z = at; at += dm;
+    L.T = at; at += dm;
+    L.S = at; at += mm;
+    L.W = at; at += mm;
+    L.X = at; at += mm;
+    L.theta = at; at += align_up((size_t)L.m * 8, kAlign);
+    L.resid = at; at += align_up((size_t)L.m * 8, kAlign);
+    L.scal = at; at += kAlign;
+    L.dead = at; at += align_up((size_t)L.m * 4, kAlign);
+    L.gram_scratch = at; at += umma_gram_scratch_bytes(D);
+    L.total = at;
+    return L;
+}
+
+template <typename T> __device__ __forceinline__ double to_double(T x);
+template <> __device__ __forceinline__ double to_double<double>(double x) { return x; }
+template <> __device__ __forceinline__ double to_double<float>(float x) { return (double)x; }
+template <> __device__ __forceinline__ double to_double<__nv_bfloat16>(__nv_bfloat16 x) {
+    return (double)__bfloat162float(x);
+}
+
+// ---------------------------------------------------------------------------------------
+// fp64 GEMM on the plain ALUs:  C[i][j] (+)= sum_l A(l, i) * B[l][j],  i < Md, j < Nd, l < L.
+//   A_T = true :  A(l, i) = A[l * lda + i]     ("TN": the reduction index is the row of A)
+//   A_T = false:  A(l, i) = A[i * lda + l]     ("NN")
+// 64 x 64 tile of C per CTA, 4 x 4 outputs per thread, 16-deep shared-memory slabs.
+// upper_only: only tiles with tj >= ti are computed (C symmetric, mirrored later).
+// ---------------------------------------------------------------------------------------
+constexpr int GT = 64, GK = 16;
+
+template <typename TA, typename TB, bool A_T>
+__global__ void __launch_bounds__(256)
+dgemm_kernel(const TA *__restrict__ A, int64_t lda, const TB *__restrict__ B, int64_t ldb, double *C,
+             int64_t ldc, int Md, int Nd, int64_t L, int accumulate, int upper_only) {
+    __shared__ double As[GK][GT + 2];
+    __shared__ double Bs[GK][GT + 2];
+    int ti, tj;
+    if (upper_only) {
+        const int nt = (Md + GT - 1) / GT;
+        int rem = blockIdx.x;
+        ti = 0;
+        while (rem >= nt - ti) { rem -= nt - ti; ++ti; }
+        tj = ti + rem;
+    } else {
+        const int ntj = (Nd + GT - 1) / GT;
+        ti = blockIdx.x / ntj;
+        tj = blockIdx.x % ntj;
+    }
+    const int i0 = ti * GT, j0 = tj * GT;
+    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
+    double acc[4][4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
+
+    for (int64_t l0 = 0; l0 < L; l0 += GK) {
+        for (int e = threadIdx.x; e < GK * GT; e += 256) {
+            int kk, ii;
+            if (A_T) { kk = e / GT; ii = e % GT; } else { ii = e / GK; kk = e % GK; }
+            const int64_t l = l0 + kk;
+            const int i = i0 + ii;
+            double v = 0.0;
+            if (l < L && i < Md) v = to_double(A_T ? A[l * lda + i] : A[(int64_t)i * lda + l]);
+            As[kk][ii] = v;
+        }
+        for (int e = threadIdx.x; e < GK * GT; e += 256) {
+            const int kk = e / GT, jj = e % GT;
+            const int64_t l = l0 + kk;
+            const int j = j0 + jj;
+            Bs[kk][jj] = (l < L && j < Nd) ? to_double(B[l * ldb + j]) : 0.0;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < GK; ++kk) {
+            double a[4], b[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { a[u] = As[kk][ty * 4 + u]; b[u] = Bs[kk][tx * 4 + u]; }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int v = 0; v < 4; ++v) acc[u][v] = fma(a[u], b[v], acc[u][v]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const int i = i0 + ty * 4 + u;
+        if (i >= Md) continue;
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            const int j = j0 + tx * 4 + v;
+            if (j >= Nd) continue;
+            double *c = C + (int64_t)i * ldc + j;
+            *c = accumulate ? (*c + acc[u][v]) : acc[u][v];
+        }
+    }
+}
+
+template <typename TA, typename TB, bool A_T>
+int dgemm(const TA *A, int64_t lda, const TB *B, int64_t ldb, double *C, int64_t ldc, int Md, int Nd,
+          int64_t L, bool accumulate, bool upper_only, cudaStream_t s) {
+    const int nti = (Md + GT - 1) / GT, ntj = (Nd + GT - 1) / GT;
+    const int blocks = upper_only ? nti * (nti + 1) / 2 : nti * ntj;
+    dgemm_kernel<TA, TB, A_T><<<blocks, 256, 0, s>>>(A, lda, B, ldb, C, ldc, Md, Nd, L, accumulate ? 1 : 0,
+                                                     upper_only ? 1 : 0);
+    count_launch();
+    return check_last_launch();
+}
+
+__global__ void zero_kernel(double *p, int64_t n) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        p[i] = 0.0;
+}
+
+__global__ void init_header_kernel(CalibHeader *h, int D, int k) {
+    h->D = D; h->k_max = k; h->rows = 0;
+}
+
+__global__ void add_rows_kernel(CalibHeader *h, int64_t M) { h->rows += M; }
+
+// lower <- upper (mode 0), or S <- (S + S^T)/2 (mode 1)
+__global__ void symmetrize_kernel(double *A, int n, int mode) {
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < (int64_t)n * n;
+         e += (int64_t)gridDim.x * blockDim.x) {
+        const int i = (int)(e / n), j = (int)(e % n);
+        if (j < i) {
+            if (mode == 0) {
+                A[(int64_t)i * n + j] = A[(int64_t)j * n + i];
+            } else {
+                const double v = 0.5 * (A[(int64_t)i * n + j] + A[(int64_t)j * n + i]);
+                A[(int64_t)i * n + j] = v;
+                A[(int64_t)j * n + i] = v;
+            }
+        }
+    }
+}
+
+__global__ void trace_kernel(const double *G, int n, double *out) {
+    __shared__ double red[256];
+    double s = 0.0;
+    for (int i = threadIdx.x; i < n; i += 256) s += G[(int64_t)i * n + i];
+    red[threadIdx.x] = s;
+    __syncthreads();
+    for (int w = 128; w > 0; w >>= 1) {
+        if (threadIdx.x < w) red[threadIdx.x] += red[threadIdx.x + w];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *out = red[0];
+}
+
+__device__ __forceinline__ uint64_t mix64(uint64_t z) {
+    z += 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+// start block: entries uniform in (-1, 1) from a counter hash (deterministic)
+__global__ void init_block_kernel(double *Q, int64_t n) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        Q[i] = (double)(mix64((uint64_t)i) >> 11) * (2.0 / 9007199254740992.0) - 1.0;
+}
+
+// ---------------------------------------------------------------------------------------
+// Cholesky-QR helper on the m x m Gram matrix S = Z^T Z of a block (one CTA):
+//   d_j = 1/sqrt(S_jj);  S' = d S d (unit diagonal);  S' = L L^T;  XT = d L^-T,
+// so that Z XT has orthonormal columns.  Scaling first makes the factorisation depend on
+// the angles between the columns only, not on their norms (which span lambda_1..lambda_m).
+// A column that is numerically dependent on the ones before it (scaled pivot <= 1e-10)
+// or is zero is marked dead: its output column is zero and the caller re-seeds it.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024) chol_inv_kernel(double *S, double *XT, int m, int *dead) {
+    __shared__ double s_dinv[384];
+    __shared__ int s_dead[384];
+    __shared__ double s_d;
+    const int tid = threadIdx.x, nt = blockDim.x;
+    for (int j = tid; j < m; j += nt) {
+        const double p = S[(int64_t)j * m + j];
+        const bool ok = (p > 0.0) && isfinite(p);
+        s_dinv[j] = ok ? 1.0 / sqrt(p) : 0.0;
+        s_dead[j] = ok ? 0 : 1;
+    }
+    __syncthreads();
+    for (int e = tid; e < m * m; e += nt) {
+        const int i = e / m, j = e % m;
+        S[e] = S[e] * s_dinv[i] * s_dinv[j];
+    }
+    __syncthreads();
+    for (int j = 0; j < m; ++j) {
+        if (tid == 0) {
+            const double p = S[(int64_t)j * m + j];
+            if (s_dead[j] || !(p > 1e-10)) { s_dead[j] = 1; s_d = 0.0; S[(int64_t)j * m + j] = 1.0; }
+            else { s_d = sqrt(p); S[(int64_t)j * m + j] = s_d; }
+        }
+        __syncthreads();
+        const double d = s_d;
+        if (d == 0.0) {   // dead column: no coupling to the rest
+            for (int i = j + 1 + tid; i < m; i += nt) S[(int64_t)i * m + j] = 0.0;
+            __syncthreads();
+            continue;
+        }
+        const double inv = 1.0 / d;
+        for (int i = j + 1 + tid; i < m; i += nt) S[(int64_t)i * m + j] *= inv;
+        __syncthreads();
+        // trailing update of the lower triangle: S[i][l] -= L[i][j] L[l][j], j < l <= i
+        const int rem = m - j - 1;
+        for (int e = tid; e < rem * rem; e += nt) {
+            const int i = j + 1 + e / rem, l = j + 1 + e % rem;
+            if (l <= i) S[(int64_t)i * m + l] -= S[(int64_t)i * m + j] * S[(int64_t)l * m + j];
+        }
+        __syncthreads();
+    }
+    // X = L^-1 by forward substitution, one column c per thread, stored as row c of XT
+    for (int c = tid; c < m; c += nt) {
+        for (int i = 0; i < c; ++i) XT[(int64_t)c * m + i] = 0.0;
+        XT[(int64_t)c * m + c] = 1.0 / S[(int64_t)c * m + c];
+        for (int i = c + 1; i < m; ++i) {
+            double acc = 0.0;
+            for (int l = c; l < i; ++l) acc += S[(int64_t)i * m + l] * XT[(int64_t)c * m + l];
+            XT[(int64_t)c * m + i] = -acc / S[(int64_t)i * m + i];
+        }
+    }
+    __syncthreads();
+    // XT[l][j] = d_l * X[j][l]; dead output columns are zeroed
+    for (int e = tid; e < m * m; e += nt) {
+        const int l = e / m, j = e % m;
+        XT[e] = s_dead[j] ? 0.0 : XT[e] * s_dinv[l];
+    }
+    for (int j = tid; j < m; j += nt) dead[j] = s_dead[j];
+}
+// Indexing: XT[c][i] holds X[i][c] = (L^-1)[i][c], i.e. (L^-T)[c][i]; the product Z XT
+// reads B[l][j] = XT[l][j] = d_l (L^-T)[l][j].
+
+// fresh pseudo-random entries for the columns marked dead (salted by `salt`)
+__global__ void reseed_dead_kernel(double *Q, int D, int m, const int *dead, uint64_t salt) {
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < (int64_t)D * m;
+         e += (int64_t)gridDim.x * blockDim.x) {
+        const int j = (int)(e % m);
+        if (dead[j]) Q[e] = (double)(mix64((uint64_t)e ^ (salt * 0x9E3779B97F4A7C15ull)) >> 11) * (2.0 / 9007199254740992.0) - 1.0;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Eigen-decomposition of the m x m symmetric Rayleigh-Ritz matrix by parallel cyclic
+// Jacobi (round-robin ordering: m/2 disjoint plane rotations per round).  One CTA.
+//   S   in: symmetric matrix (destroyed)     W   scratch m x m
+//   Wout out: eigenvectors as columns, ordered by descending eigenvalue
+//   theta out: eigenvalues, descending       sweeps_out: sweeps used
+// A round applies J^T S J for J = product of the round's rotations: the 2 x 2 block of S
+// that pairs rotation A's rows with rotation B's columns becomes J_A^T S_AB J_B, so all
+// (m/2)^2 blocks update independently.  m must be even.
+// ---------------------------------------------------------------------------------------
+constexpr int kMaxRitz = 384;
+
+__global__ void __launch_bounds__(1024)
+jacobi_kernel(double *S, double *W, double *Wout, double *theta, int m, double *sweeps_out) {
+    __shared__ double cs_c[kMaxRitz / 2], cs_s[kMaxRitz / 2];
+    __shared__ int pr_p[kMaxRitz / 2], pr_q[kMaxRitz / 2];
+    __shared__ int s_rot;
+    __shared__ double s_diag[kMaxRitz];
+    __shared__ int s_rank[kMaxRitz];
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int h = m / 2;
+    for (int e = tid; e < m * m; e += nt) W[e] = (e / m == e % m) ? 1.0 : 0.0;
+    __syncthreads();
+    int sweep = 0;
+    for (; sweep < 40; ++sweep) {
+        if (tid == 0) s_rot = 0;
+        __syncthreads();
+        for (int r = 0; r < m - 1; ++r) {
+            if (tid < h) {
+                int p, q;
+                if (tid == 0) { p = m - 1; q = r; }
+                else { p = (r + tid) % (m - 1); q = (r - tid + (m - 1)) % (m - 1); }
+                if (p > q) { const int t = p; p = q; q = t; }
+                pr_p[tid] = p; pr_q[tid] = q;
+                const double app = S[(int64_t)p * m + p], aqq = S[(int64_t)q * m + q], apq = S[(int64_t)p * m + q];
+                double c = 1.0, s = 0.0;
+                if (apq != 0.0 && fabs(apq) > 1e-17 * sqrt(fabs(app * aqq)) ) {
+                    const double tau = (aqq - app) / (2.0 * apq);
+                    const double t = (tau >= 0.0 ? 1.0 : -1.0) / (fabs(tau) + sqrt(1.0 + tau * tau));
+                    c = 1.0 / sqrt(1.0 + t * t);
+                    s = t * c;
+                    if (fabs(apq) > 1e-15 * sqrt(fabs(app * aqq))) atomicAdd(&s_rot, 1);
+                }
+                cs_c[tid] = c; cs_s[tid] = s;
+            }
+            __syncthreads();
+            // S_AB <- J_A^T S_AB J_B with J = [[c, s], [-s, c]] on the (p, q) plane
+            for (int e = tid; e < h * h; e += nt) {
+                const int A = e / h, B = e % h;
+                const int p = pr_p[A], q = pr_q[A], u = pr_p[B], v = pr_q[B];
+                const double ca = cs_c[A], sa = cs_s[A], cb = cs_c[B], sb = cs_s[B];
+                double spu = S[(int64_t)p * m + u], spv = S[(int64_t)p * m + v];
+                double squ = S[(int64_t)q * m + u], sqv = S[(int64_t)q * m + v];
+                // rows: (p, q) <- (c p - s q, s p + c q)
+                const double rpu = ca * spu - sa * squ, rpv = ca * spv - sa * sqv;
+                const double rqu = sa * spu + ca * squ, rqv = sa * spv + ca * sqv;
+                // columns: (u, v) <- (c u - s v, s u + c v)
+                S[(int64_t)p * m + u] = cb * rpu - sb * rpv;
+                S[(int64_t)p * m + v] = sb * rpu + cb * rpv;
+                S[(int64_t)q * m + u] = cb * rqu - sb * rqv;
+                S[(int64_t)q * m + v] = sb * rqu + cb * rqv;
+            }
+            // W <- W J (columns)
+            for (int e = tid; e < m * h; e += nt) {
+                const int i = e / h, B = e % h;
+                const int u = pr_p[B], v = pr_q[B];
+                const double cb = cs_c[B], sb = cs_s[B];
+                const double wu = W[(int64_t)i * m + u], wv = W[(int64_t)i * m + v];
+                W[(int64_t)i * m + u] = cb * wu - sb * wv;
+                W[(int64_t)i * m + v] = sb * wu + cb * wv;
+            }
+            __syncthreads();
+        }
+        if (s_rot == 0) { ++sweep; break; }
+        __syncthreads();
+    }
+    // order by descending eigenvalue (rank sort; ties by index)
+    for (int i = tid; i < m; i += nt) s_diag[i] = S[(int64_t)i * m + i];
+    __syncthreads();
+    for (int j = tid; j < m; j += nt) {
+        int rk = 0;
+        const double x = s_diag[j];
+        for (int i = 0; i < m; ++i) rk += (s_diag[i] > x) || (s_diag[i] == x && i < j);
+        s_rank[j] = rk;
+        theta[rk] = x;
+    }
+    __syncthreads();
+    for (int e = tid; e < m * m; e += nt) {
+        const int i = e / m, j = e % m;
+        Wout[(int64_t)i * m + s_rank[j]] = W[e];
+    }
+    if (tid == 0 && sweeps_out) *sweeps_out = (double)sweep;
+}
+
+// resid[j] = | Z[:, j] - theta[j] Q[:, j] |_2  for j < k;  one CTA per column
+__global__ void residual_kernel(const double *Z, const double *Q, const double *theta, int D, int m,
+                                double *resid) {
+    __shared__ double red[256];
+    const int j = blockIdx.x;
+    const double th = theta[j];
+    double s = 0.0;
+    for (int i = threadIdx.x; i < D; i += 256) {
+        const double r = Z[(int64_t)i * m + j] - th * Q[(int64_t)i * m + j];
+        s += r * r;
+    }
+    red[threadIdx.x] = s;
+    __syncthreads();
+    for (int w = 128; w > 0; w >>= 1) {
+        if (threadIdx.x < w) red[threadIdx.x] += red[threadIdx.x + w];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) resid[j] = sqrt(red[0]);
+}
+
+// scal[1] = max_j resid[j] / max(theta[0], tiny)
+__global__ void max_residual_kernel(const double *resid, const double *theta, int k, double *scal) {
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        double mx = 0.0;
+        for (int j = 0; j < k; ++j) mx = fmax(mx, resid[j]);
+        const double t0 = fabs(theta[0]);
+        scal[1] = (t0 > 0.0) ? mx / t0 : 0.0;
+    }
+}
+
+// V_k (fp32) <- first k columns of Q with the sign convention; lambda <- theta[:k]
+__global__ void emit_basis_kernel(const double *Q, const double *theta, int D, int m, int k, float *Vk,
+                                  double *lambda) {
+    __shared__ double best_abs[256];
+    __shared__ double best_val[256];
+    const int j = blockIdx.x;
+    double ba = -1.0, bv = 0.0;
+    for (int i = threadIdx.x; i < D; i += 256) {   // first index of the largest magnitude
+        const double v = Q[(int64_t)i * m + j];
+        if (fabs(v) > ba) { ba = fabs(v); bv = v; }
+    }
+    best_abs[threadIdx.x] = ba;
+    best_val[threadIdx.x] = bv;
+    __syncthreads();
+    for (int w = 128; w > 0; w >>= 1) {
+        if (threadIdx.x < w && best_abs[threadIdx.x + w] > best_abs[threadIdx.x]) {
+            best_abs[threadIdx.x] = best_abs[threadIdx.x + w];
+            best_val[threadIdx.x] = best_val[threadIdx.x + w];
+        }
+        __syncthreads();
+    }
+    const double sgn = (best_val[0] < 0.0) ? -1.0 : 1.0;
+    for (int i = threadIdx.x; i < D; i += 256) Vk[(int64_t)i * k + j] = (float)(sgn * Q[(int64_t)i * m + j]);
+    if (threadIdx.x == 0 && lambda) lambda[j] = theta[j];
+}
+
+__global__ void copy_scalar_kernel(const double *src, double *dst) { *dst = *src; }
+
+int grid_for(int64_t n) { return (int)std::min<int64_t>((n + 255) / 256, 148 * 8); }
+
+}  // namespace
+
+size_t calib_workspace_bytes(int D, int k) { return calib_layout(D, k).total; }
+
+int calib_begin(int D, int k, void *ws, cudaStream_t s) {
+    const CalibLayout L = calib_layout(D, k);
+    char *w = (char *)ws;
+    init_header_kernel<<<1, 1, 0, s>>>((CalibHeader *)w, D, k);
+    zero_kernel<<<grid_for((int64_t)D * D), 256, 0, s>>>((double *)(w + L.G), (int64_t)D * D);
+    count_launch(2);
+    return check_last_launch();
+}
+
+int calib_accumulate(const void *F, int64_t M, int D, int64_t ld, int dtype, void *ws, cudaStream_t s) {
+    // G sits at a fixed offset whatever k is
+    char *w = (char *)ws;
+    double *G = (double *)(w + kHeaderBytes);
+    int rc;
+    if (umma_gram_supported(M, D, ld, dtype)) {
+        const CalibLayout L = calib_layout(D, 8);
+        rc = umma_gram_accumulate(F, M, D, ld, G, w + L.gram_scratch, umma_gram_scratch_bytes(D), s);
+    } else if (dtype == SVDCACHE_BF16) {
+        const __nv_bfloat16 *f = (const __nv_bfloat16 *)F;
+        rc = dgemm<__nv_bfloat16, __nv_bfloat16, true>(f, ld, f, ld, G, D, D, D, M, true, true, s);
+    } else {
+        const float *f = (const float *)F;
+        rc = dgemm<float, float, true>(f, ld, f, ld, G, D, D, D, M, true, true, s);
+    }
+    if (rc) return rc;
+    add_rows_kernel<<<1, 1, 0, s>>>((CalibHeader *)w, M);
+    count_launch();
+    return check_last_launch();
+}
+
+namespace {
+
+// Q (D x m) <- orthonormal basis of the columns of Zin (scaled Cholesky-QR, twice; columns
+// found dependent in the first pass are re-seeded before the second).  Zin is destroyed;
+// T is scratch.  The result ends up in Zin's buffer, returned through *out.
+int orthonormalize(double *Zin, double *T, double *S, double *X, int *dead, int D, int m, uint64_t salt,
+                   double **out, cudaStream_t s) {
+    double *src = Zin, *dst = T;
+    for (int pass = 0; pass < 2; ++pass) {
+        int rc = dgemm<double, double, true>(src, m, src, m, S, m, m, m, D, false, false, s);
+        if (rc) return rc;
+        symmetrize_kernel<<<grid_for((int64_t)m * m), 256, 0, s>>>(S, m, 1);
+        chol_inv_kernel<<<1, 1024, 0, s>>>(S, X, m, dead);
+        count_launch(2);
+        rc = dgemm<double, double, false>(src, m, X, m, dst, m, D, m, m, false, false, s);
+        if (rc) return rc;
+        if (pass == 0) {
+            reseed_dead_kernel<<<grid_for((int64_t)D * m), 256, 0, s>>>(dst, D, m, dead, salt);
+            count_launch();
+        }
+        std::swap(src, dst);
+    }
+    *out = src;
+    return check_last_launch();
+}
+
+}  // namespace
+
+int calib_finish(int D, int k, float *Vk, double *lambda, double *trace, double *info, void *ws,
+                 cudaStream_t s) {
+    const CalibLayout L = calib_layout(D, k);
+    const int m = L.m;
+    if (m > kMaxRitz || (m % 2) != 0) return SVDCACHE_ERR_BAD_SHAPE;
+    char *w = (char *)ws;
+    double *G = (double *)(w + L.G);
+    double *bufA = (double *)(w + L.Q), *bufB = (double *)(w + L.Z), *bufC = (double *)(w + L.T);
+    double *S = (double *)(w + L.S), *W = (double *)(w + L.W), *X = (double *)(w + L.X);
+    double *theta = (double *)(w + L.theta), *resid = (double *)(w + L.resid), *scal = (double *)(w + L.scal);
+    // scal[0] = trace, scal[1] = max relative residual, scal[2] = Jacobi sweeps
+
+    symmetrize_kernel<<<grid_for((int64_t)D * D), 256, 0, s>>>(G, D, 0);
+    trace_kernel<<<1, 256, 0, s>>>(G, D, scal);
+    init_block_kernel<<<grid_for((int64_t)D * m), 256, 0, s>>>(bufA, (int64_t)D * m);
+    count_launch(3);
+    int rc = check_last_launch();
+    if (rc) return rc;
+
+    int *dead = (int *)(w + L.dead);
+    double *Q = nullptr;
+    rc = orthonormalize(bufA, bufB, S, X, dead, D, m, 1, &Q, s);
+    if (rc) return rc;
+    auto others = [&](double *q, double **z, double **t) {
+        double *all[3] = {bufA, bufB, bufC};
+        int n = 0;
+        double *o[2];
+        for (double *b : all)
+            if (b != q) o[n++] = b;
+        *z = o[0]; *t = o[1];
+    };
+
+    // Every iteration: Z = G Q; Rayleigh-Ritz on span(Q) (S = Q^T Z = W Theta W^T, Q <- Q W,
+    // Z <- Z W); residual check; Q <- orthonormalise(Z).  The Ritz rotation keeps the columns
+    // of Z close to mutually orthogonal, which is what the scaled Cholesky-QR relies on.
+    const double tol = 1e-12;
+    const int max_mult = 200;
+    double max_rel = 1.0;
+    int mult = 0;
+    bool converged = false;
+    while (mult < max_mult) {
+        double *Z, *T;
+        others(Q, &Z, &T);
+        rc = dgemm<double, double, true>(G, D, Q, m, Z, m, D, m, D, false, false, s);   // Z = G Q
+        if (rc) return rc;
+        ++mult;
+        rc = dgemm<double, double, true>(Q, m, Z, m, S, m, m, m, D, false, false, s);   // S = Q^T Z
+        if (rc) return rc;
+        symmetrize_kernel<<<grid_for((int64_t)m * m), 256, 0, s>>>(S, m, 1);
+        jacobi_kernel<<<1, 1024, 0, s>>>(S, X, W, theta, m, scal + 2);
+        count_launch(2);
+        rc = dgemm<double, double, false>(Q, m, W, m, T, m, D, m, m, false, false, s);  // ritz = Q W
+        if (rc) return rc;
+        rc = dgemm<double, double, false>(Z, m, W, m, Q, m, D, m, m, false, false, s);  // image = Z W
+        if (rc) return rc;
+        double *ritz = T, *image = Q;   // `Z` is free scratch from here on
+        const bool check = (mult >= 4 && (mult % 2) == 0) || mult == max_mult;
+        if (check) {
+            residual_kernel<<<k, 256, 0, s>>>(image, ritz, theta, D, m, resid);
+            max_residual_kernel<<<1, 32, 0, s>>>(resid, theta, k, scal);
+            count_launch(2);
+            rc = record_cuda(cudaMemcpyAsync(&max_rel, scal + 1, sizeof(double), cudaMemcpyDeviceToHost, s));
+            if (rc) return rc;
+            rc = record_cuda(cudaStreamSynchronize(s));
+            if (rc) return rc;
+            if (max_rel <= tol || mult == max_mult) {
+                converged = max_rel <= tol;
+                Q = ritz;
+                break;
+            }
+        }
+        rc = orthonormalize(image, Z, S, X, dead, D, m, (uint64_t)mult + 1, &Q, s);
+        if (rc) return rc;
+    }
+
+    emit_basis_kernel<<<k, 256, 0, s>>>(Q, theta, D, m, k, Vk, lambda);
+    count_launch();
+    if (trace) {
+        copy_scalar_kernel<<<1, 1, 0, s>>>(scal, trace);
+        count_launch();
+    }
+    rc = check_last_launch();
+    if (rc) return rc;
+    double sweeps = 0.0;
+    rc = record_cuda(cudaMemcpyAsync(&sweeps, scal + 2, sizeof(double), cudaMemcpyDeviceToHost, s));
+    if (rc) return rc;
+    rc = record_cuda(cudaStreamSynchronize(s));
+    if (rc) return rc;
+    if (info) {
+        info[0] = (double)mult;
+        info[1] = max_rel;
+        info[2] = (double)m;
+        info[3] = sweeps;
+    }
+    return converged ? SVDCACHE_OK : SVDCACHE_ERR_NOT_CONVERGED;
+}
+
+}  // namespace svdc

@@ -1,0 +1,135 @@
+"""GPU parity of the calibration path (Gram matrix + top-k eigenvectors, Eq. 4 - Eq. 7)
+against the fp64 oracle on the same seeded stacks, through the C ABI.
+
+Several bases are correct for one stack (signs, and rotations inside near-degenerate
+eigenvalue clusters), so the basis is compared through what is unique: the principal
+angles between the two k-dimensional subspaces, the eigenvalues and the trace."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import svdcache_oracle as oracle
+from paper_2601_07396_b200 import binding as sc
+from paper_2601_07396_b200 import streams
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+COS_MIN = 1.0 - 1e-4
+
+
+def _compare(stack: torch.Tensor, k: int, Vk, lam, tr, check_gap=True):
+    Fh = stack.double().cpu().numpy()
+    Vo, lo, to, lall = oracle.calibrate(Fh, k, all_eigenvalues=True)
+    V = Vk.double().cpu().numpy()
+    lam = lam.cpu().numpy()
+    # orthonormal (fp32 storage), ordered, signed
+    np.testing.assert_allclose(V.T @ V, np.eye(k), atol=5e-6)
+    assert np.all(np.diff(lam) <= 1e-12 * lam[0])
+    assert np.all(V[np.argmax(np.abs(V), axis=0), np.arange(k)] > 0)
+    # eigenvalues and trace
+    np.testing.assert_allclose(lam, lo, rtol=1e-9, atol=1e-12 * lo[0])
+    assert float(tr.cpu()[0]) == pytest.approx(to, rel=1e-12)
+    # the subspace is well defined only if lambda_k is separated from lambda_{k+1}
+    if check_gap and k < len(lall):
+        gap = (lall[k - 1] - lall[k]) / lall[k - 1]
+        assert gap > 1e-3, f"oracle eigen-gap at k too small to grade angles: {gap:.2e}"
+    cos = np.linalg.svd(Vo.T @ V, compute_uv=False)
+    assert cos.min() >= COS_MIN, f"smallest principal-angle cosine {cos.min():.8f}"
+    return cos.min()
+
+
+def test_tiny_config_calibration():
+    spec = streams.TINY
+    stack = streams.calibration_stack(spec, 0, device=DEV)
+    assert stack.shape == (4096, 1152) and stack.dtype == torch.float32
+    Vk, lam, tr, info = sc.svdcache_calibrate(stack, spec.k)
+    _compare(stack, spec.k, Vk, lam, tr)
+    assert info[1] <= 1e-12
+
+
+@pytest.mark.parametrize("block", [0, 27])
+def test_dit_xl_config_calibration(block):
+    spec = streams.DIT_XL
+    # 16 calibration trajectories x 4 timesteps x 256 tokens (batch 1) = 16,384 rows
+    stack = streams.calibration_stack(spec, block, device=DEV, rows_per_snapshot=256)
+    assert stack.shape == (16384, 1152) and stack.dtype == torch.bfloat16
+    Vk, lam, tr, info = sc.svdcache_calibrate(stack, spec.k)
+    _compare(stack, spec.k, Vk, lam, tr)
+
+
+def test_flux_width_calibration_single_snapshot():
+    """FLUX width (D = 3072) on one snapshot of 4608 rows (the smallest stack of the
+    calibration sweep); the full 294,912-row stack differs only in the Gram loop length."""
+    spec = streams.FLUX
+    stack = streams.calibration_stack(spec, 0, device=DEV, trajectories=(1,), timesteps=(0,))
+    assert stack.shape == (4608, 3072)
+    Vk, lam, tr, info = sc.svdcache_calibrate(stack, spec.k)
+    _compare(stack, spec.k, Vk, lam, tr)
+
+
+@pytest.mark.parametrize("M,D,k,dtype", [(100, 64, 8, "f32"), (1000, 264, 24, "bf16"), (37, 128, 16, "f32"),
+                                         (5000, 512, 256, "bf16"), (3001, 1000, 128, "bf16")])
+def test_ragged_shapes(M, D, k, dtype):
+    spec = streams.StreamSpec("cal", blocks=1, rows=M, D=D, dtype=dtype, k=k, T=2, interval=1,
+                              rank=min(D, max(2 * k, 48)), amp=40.0, power=1.0, noise_std=0.02)
+    stack = streams.BlockStream(spec, 0, device=DEV).features(1)
+    Vk, lam, tr, info = sc.svdcache_calibrate(stack, k)
+    _compare(stack, k, Vk, lam, tr, check_gap=(M > k))
+
+
+def test_streaming_accumulation_matches_one_shot():
+    spec = streams.StreamSpec("cal", blocks=1, rows=3000, D=384, dtype="bf16", k=32, T=2, interval=1,
+                              rank=96, amp=40.0, power=1.1, noise_std=0.02)
+    stack = streams.BlockStream(spec, 0, device=DEV).features(0)
+    ws = torch.empty(sc.svdcache_calibrate_workspace_bytes(384, 32), dtype=torch.uint8, device=DEV)
+    sc.svdcache_calibrate_begin(384, 32, ws)
+    for lo, hi in ((0, 1), (1, 1000), (1000, 1000), (1000, 2999), (2999, 3000)):
+        sc.svdcache_calibrate_accumulate(stack[lo:hi], ws)
+    Vk, lam, tr, info = sc.svdcache_calibrate_finish(384, 32, ws)
+    _compare(stack, 32, Vk, lam, tr)
+    # and the run is reproducible bit for bit
+    sc.svdcache_calibrate_begin(384, 32, ws)
+    for lo, hi in ((0, 1), (1, 1000), (1000, 1000), (1000, 2999), (2999, 3000)):
+        sc.svdcache_calibrate_accumulate(stack[lo:hi], ws)
+    Vk2, lam2, tr2, _ = sc.svdcache_calibrate_finish(384, 32, ws)
+    assert torch.equal(Vk, Vk2) and torch.equal(lam, lam2) and torch.equal(tr, tr2)
+
+
+def test_noise_free_stack_recovers_the_generator_basis():
+    spec = streams.StreamSpec("cal", blocks=1, rows=2000, D=256, dtype="f32", k=16, T=2, interval=1,
+                              rank=16, amp=10.0, power=0.5, noise_std=0.0)
+    st = streams.BlockStream(spec, 0, device=DEV)
+    stack = st.features(0)
+    Vk, lam, tr, info = sc.svdcache_calibrate(stack, 16, strict=False)
+    cos = torch.linalg.svdvals(st.V_gen.t() @ Vk.double())
+    assert float(cos.min()) >= 1 - 1e-6
+    assert float(lam.sum()) == pytest.approx(float(tr[0]), rel=1e-6)   # all the energy is in rank 16
+
+
+def test_rank_selection_by_energy_threshold():
+    """Eq. 6 on the calibrated spectrum, against the oracle's rule."""
+    spec = streams.TINY
+    stack = streams.calibration_stack(spec, 0, device=DEV)
+    Vk, lam, tr, _ = sc.svdcache_calibrate(stack, 64)
+    lam_h, tr_h = lam.cpu().numpy(), float(tr.cpu()[0])
+    for tau in (0.5, 0.85, 0.9, 0.99):
+        assert sc.svdcache_rank_for_energy(lam_h, tr_h, tau) == oracle.rank_for_energy(lam_h, tr_h, tau)
+    assert 1 <= sc.svdcache_rank_for_energy(lam_h, tr_h, 0.85) < 64
+
+
+def test_calibration_argument_errors():
+    L = sc.lib()
+    ws = torch.empty(sc.svdcache_calibrate_workspace_bytes(64, 8), dtype=torch.uint8, device=DEV)
+    F = torch.zeros(16, 64, device=DEV)
+    p = lambda t: ctypes.c_void_p(t.data_ptr())
+    s = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    assert L.svdcache_calibrate_begin(64, 8, p(ws), 100, s) == -5
+    assert L.svdcache_calibrate_begin(64, 9, p(ws), ws.numel(), s) == -2
+    assert L.svdcache_calibrate_begin(64, 8, None, ws.numel(), s) == -1
+    assert L.svdcache_calibrate_begin(64, 8, ctypes.c_void_p(ws.data_ptr() + 16), ws.numel() - 16, s) == -3
+    assert L.svdcache_calibrate_accumulate(p(F), 16, 64, 60, 0, p(ws), ws.numel(), s) == -2
+    assert L.svdcache_calibrate_accumulate(p(F), 16, 64, 64, 3, p(ws), ws.numel(), s) == -1
+    assert L.svdcache_calibrate(p(F), 0, 64, 64, 0, 8, p(F), None, None, None, p(ws), ws.numel(), s) == -2
+    torch.cuda.synchronize()
