@@ -126,7 +126,11 @@ SVDCACHE_API int svdcache_basis_prepare(const float *Vk, int D, int k, int dtype
 
 /* ---------------------------------------------------------------------------------
  * Per-block cache state, a caller-owned flat device buffer (checkpoint = memcpy):
- *   header (256 B) | Chat fp32 [N x k] | R dtype [N x D]          (dense, no pitch)
+ *   header (256 B) | Chat fp32 [N x k] | Chat operand copy | R dtype [N x D]   (dense, no pitch)
+ * The operand copy exists only for dtype = SVDCACHE_BF16: Chat as two bf16 arrays [N x k],
+ * hi = bf16(Chat) and lo = bf16(Chat - hi), which every full step rewrites together with
+ * Chat and the cached step feeds to the tensor cores as they are (hi + lo carries ~16
+ * mantissa bits).  Offsets of Chat and R come from svdcache_state_layout.
  * The header counts the full steps the state has seen and carries a sticky device
  * status word.  svdcache_state_reset must be called once before first use (and again to
  * start a new sampling run): it clears the counter, so the next full step initialises

@@ -15,7 +15,9 @@ F32, BF16 = 0, 1
 _DTYPES = {torch.float32: F32, torch.bfloat16: BF16}
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libsvdcache.so")
+# SVDCACHE_LIBRARY names another build of the same library (e.g. one made with different
+# compiler flags); by default the in-tree build next to this file is loaded.
+LIB_PATH = os.environ.get("SVDCACHE_LIBRARY") or os.path.join(_HERE, "libsvdcache.so")
 _lib = None
 
 _vp, _i64, _ci, _sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t

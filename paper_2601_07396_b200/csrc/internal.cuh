@@ -48,15 +48,27 @@ inline BasisLayout basis_layout(int D, int k, int dtype) {
     return L;
 }
 
+// header | Chat fp32 [N x k] | (bf16 only) Chat as a split-bf16 pair: hi [N x k], lo [N x k] |
+// R [N x D].  hi = bf16(Chat), lo = bf16(Chat - hi): the tensor-core operand of the cached
+// step, written by the full step next to Chat so that the cached step reads it as it is.
 struct StateLayout {
-    size_t chat, r, total;
+    size_t chat, op_hi, op_lo, r, total;
 };
 inline StateLayout state_layout(int64_t N, int D, int k, int dtype) {
     StateLayout L;
+    const size_t op = dtype == SVDCACHE_BF16 ? align_up((size_t)N * k * 2, kAlign) : 0;
     L.chat = kHeaderBytes;
-    L.r = L.chat + align_up((size_t)N * k * 4, kAlign);
+    L.op_hi = L.chat + align_up((size_t)N * k * 4, kAlign);
+    L.op_lo = L.op_hi + op;
+    L.r = L.op_lo + op;
     L.total = L.r + align_up((size_t)N * D * elem_bytes(dtype), kAlign);
     return L;
+}
+
+// split of an fp32 value into the bf16 pair (hi, lo) described above
+__device__ __forceinline__ void split_bf16(float x, __nv_bfloat16 &hi, __nv_bfloat16 &lo) {
+    hi = __float2bfloat16_rn(x);
+    lo = __float2bfloat16_rn(x - __bfloat162float(hi));
 }
 
 // Arguments shared by the step kernels of every family.  Pointers are block 0's; block b

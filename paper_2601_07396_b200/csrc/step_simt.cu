@@ -27,7 +27,8 @@ constexpr int kThreads = 256;
 // Full step: Eq. 8-9 (C = F V_k), Eq. 10 (R = F - C V_k^T), Eq. 11 (EMA of C).
 template <typename T, typename BT, typename Acc, int kRows>
 __global__ void __launch_bounds__(kThreads)
-simt_full_kernel(StepArgs a, size_t v_off, size_t vt_off, size_t chat_off, size_t r_off) {
+simt_full_kernel(StepArgs a, size_t v_off, size_t vt_off, StateLayout SL) {
+    const size_t chat_off = SL.chat, r_off = SL.r;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int D = a.D, k = a.k;
     float *Fs = reinterpret_cast<float *>(smem_raw);                        // kRows x D
@@ -66,7 +67,14 @@ simt_full_kernel(StepArgs a, size_t v_off, size_t vt_off, size_t chat_off, size_
             const float c = (float)acc;
             if (C_out) C_out[n * k + j] = c;
             float *ch = Chat + n * k + j;
-            *ch = first ? c : fmaf(beta, *ch, omb * c);
+            const float ema = first ? c : fmaf(beta, *ch, omb * c);
+            *ch = ema;
+            if (SL.op_lo != SL.op_hi) {   // bf16 mode: the cached step's tensor-core operand
+                __nv_bfloat16 hi, lo;
+                split_bf16(ema, hi, lo);
+                reinterpret_cast<__nv_bfloat16 *>(state + SL.op_hi)[n * k + j] = hi;
+                reinterpret_cast<__nv_bfloat16 *>(state + SL.op_lo)[n * k + j] = lo;
+            }
         }
     }
     __syncthreads();
@@ -151,7 +159,7 @@ int launch_full(const StepArgs &a, size_t v_off, size_t vt_off, cudaStream_t s) 
     int rc = record_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     if (rc) return rc;
     dim3 grid((unsigned)((a.N + kRows - 1) / kRows), (unsigned)a.nblocks);
-    kern<<<grid, kThreads, smem, s>>>(a, v_off, vt_off, SL.chat, SL.r);
+    kern<<<grid, kThreads, smem, s>>>(a, v_off, vt_off, SL);
     count_launch();
     return check_last_launch();
 }

@@ -1,15 +1,13 @@
 // tcgen05 family of the step kernels (bf16 I/O): warp-specialised, persistent, TMA-fed.
 //
 // Both kernels stream 128-row x 64-column tiles of the big operand (R or F) through a
-// ring of shared-memory stages.  A stage holds one such tile (16 KB, 128-byte swizzled,
-// written by TMA) and the matching slice of the basis.  The tensor cores produce the
-// 128 x 64 product tile into TMEM; the epilogue warps read it back, combine it with the
-// staged tile in place and hand the tile to a TMA store.  Every global access of the big
-// operands is a TMA bulk copy; the 128 x k coefficient tile is the A operand, converted to
-// bf16 and laid out in the tensor-core's swizzled K-major format by the A-prep warps.
-//
-// Warp roles (320 threads): 0 = TMA producer, 1 = MMA issuer (+ TMEM owner),
-// 2..5 = epilogue (TMEM lane quarter = warp % 4), 6..9 = A-operand preparation.
+// ring of shared-memory slots (16 KB each, 128-byte swizzled, written by TMA).  The tensor
+// cores produce the product C V_k^T into TMEM; the epilogue warps read it back, combine it
+// with the staged tile in place and hand the tile to a TMA store.  Every global access on
+// the streaming path is a TMA bulk copy: under a saturated memory system an ordinary load
+// takes microseconds, so nothing on the critical path waits for one.  The 128 x k
+// coefficient tile is the A operand, a split-bf16 pair (hi + lo) so that the product keeps
+// ~16 mantissa bits.
 #include <cstdio>
 #include <mutex>
 
@@ -27,7 +25,8 @@ constexpr int kTileRows = 128;      // MMA M
 constexpr int kTileCols = 64;       // columns of D per stage (MMA N in the reconstruct GEMM)
 constexpr int kTileBytes = kTileRows * kTileCols * 2;   // 16 KB
 constexpr int kAccStages = 4;       // TMEM accumulator ring (64 fp32 columns each)
-constexpr int kMaxStages = 10;
+constexpr int kMaxStages = 12;
+constexpr int kMaxVSlots = 2;
 constexpr int kMaxABufs = 2;
 
 struct UmmaParams {
@@ -37,8 +36,10 @@ struct UmmaParams {
     int kb_elems, kb_bytes, nkb;         // K-block of the rank dimension: min(k, 64) elements
     int stages, a_bufs;
     uint32_t a_half_bytes, a_bytes, v_bytes, stage_bytes;
+    int gc, acc_stages, acc_cols, v_slots;   // cached step: chunks per MMA group, TMEM ring, basis ring
+    uint32_t vslice_bytes;
     char *state;
-    size_t state_stride, chat_off;
+    size_t state_stride, chat_off, ophi_off, oplo_off;
     float *C_out;
     size_t C_stride;
     float beta;
@@ -50,7 +51,7 @@ struct SmemLayout {
 
 // barrier slots (8 bytes each) after the tiles
 struct Bars {
-    uint32_t full, empty, acc_full, acc_empty, a_full, a_empty, c_full, c_done, tmem_slot, abort_flag;
+    uint32_t full, empty, acc_full, acc_empty, a_full, a_empty, c_full, c_done, v_full, v_empty, tmem_slot, abort_flag;
 };
 
 __device__ __forceinline__ Bars bars_at(uint32_t base) {
@@ -63,11 +64,13 @@ __device__ __forceinline__ Bars bars_at(uint32_t base) {
     b.a_empty = b.a_full + 8 * kMaxABufs;
     b.c_full = b.a_empty + 8 * kMaxABufs;
     b.c_done = b.c_full + 8;
-    b.tmem_slot = b.c_done + 8;
+    b.v_full = b.c_done + 8;
+    b.v_empty = b.v_full + 8 * kMaxVSlots;
+    b.tmem_slot = b.v_empty + 8 * kMaxVSlots;
     b.abort_flag = b.tmem_slot + 8;
     return b;
 }
-constexpr uint32_t kBarBytes = 8 * (2 * kMaxStages + 2 * kAccStages + 2 * kMaxABufs + 4);
+constexpr uint32_t kBarBytes = 8 * (2 * kMaxStages + 2 * kAccStages + 2 * kMaxABufs + 2 * kMaxVSlots + 4);
 
 __device__ __forceinline__ StateHeader *header_of(const UmmaParams &p, int b) {
     return reinterpret_cast<StateHeader *>(p.state + (size_t)b * p.state_stride);
@@ -160,30 +163,54 @@ __device__ __forceinline__ void issue_reconstruct_mmas(const UmmaParams &p, uint
 
 // ======================================================================================
 // Cached step (Sec. 3.5):  Fhat = Chat V_k^T + R
+//
+// A unit is one 128-row tile of one block (times a column range when the launch is too
+// small to occupy the GPU otherwise).  Its A operand -- the split-bf16 copy of Chat that the
+// full step left in the state -- arrives by TMA.  The columns are walked in groups of
+// `gc` 64-column chunks: one basis slice (gc*64 x k) per group feeds MMAs of N = gc*64
+// (few, wide instructions: a dependent MMA costs ~200 cycles whatever its N), while the R
+// tiles of the group's chunks stream through their own ring and meet the accumulator in
+// the epilogue.
+//
+// Warp roles (320 threads): 0 = TMA producer, 1 = MMA issuer (+ TMEM owner), 2..9 = two
+// epilogue groups of four warps (TMEM lane quarter = warp % 4; group g takes the chunks
+// whose running index is g modulo 2).  Each epilogue warp owns a 32-row slab of the chunk
+// from the TMEM read to its own TMA store, so the eight warps never meet at a barrier.
 // ======================================================================================
-__global__ void __launch_bounds__(kThreadsUmma, 1)
+constexpr int kThreadsCached = 320;
+constexpr int kSlabRows = 32;                              // rows one epilogue warp stores
+constexpr uint32_t kSlabBytes = kSlabRows * kTileCols * 2; // 4 KB
+
+__global__ void __launch_bounds__(kThreadsCached, 1)
 umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_constant__ CUtensorMap tm_v,
+                   const __grid_constant__ CUtensorMap tm_ahi, const __grid_constant__ CUtensorMap tm_alo,
                    const __grid_constant__ CUtensorMap tm_out, const UmmaParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t a_base0 = base;
-    const uint32_t stage0 = a_base0 + (uint32_t)p.a_bufs * p.a_bytes;
-    const Bars bar = bars_at(stage0 + (uint32_t)p.stages * p.stage_bytes);
+    const uint32_t v_base0 = a_base0 + (uint32_t)p.a_bufs * p.a_bytes;
+    const uint32_t stage0 = v_base0 + (uint32_t)p.v_slots * p.vslice_bytes;
+    const Bars bar = bars_at(stage0 + (uint32_t)p.stages * kTileBytes);
     uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
     volatile int *abort_flag = reinterpret_cast<volatile int *>(gen_base + (bar.abort_flag - base));
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(gen_base + (bar.tmem_slot - base));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t tmem_cols = kAccStages * kTileCols;   // 256
+    const uint32_t tmem_cols = 512;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < p.stages; ++s) { mbar_init(bar.full + 8 * s, 1); mbar_init(bar.empty + 8 * s, 2); }
-        for (int s = 0; s < kAccStages; ++s) { mbar_init(bar.acc_full + 8 * s, 1); mbar_init(bar.acc_empty + 8 * s, 128); }
-        for (int s = 0; s < p.a_bufs; ++s) { mbar_init(bar.a_full + 8 * s, 128); mbar_init(bar.a_empty + 8 * s, 1); }
+        // R slot: free again once the four slab stores have read it.  Accumulator: four
+        // arrivals (one per lane quarter) for each of the gc chunks of a group.
+        for (int s = 0; s < p.stages; ++s) { mbar_init(bar.full + 8 * s, 1); mbar_init(bar.empty + 8 * s, 4); }
+        for (int s = 0; s < p.acc_stages; ++s) { mbar_init(bar.acc_full + 8 * s, 1); mbar_init(bar.acc_empty + 8 * s, 4 * p.gc); }
+        for (int s = 0; s < p.a_bufs; ++s) { mbar_init(bar.a_full + 8 * s, 1); mbar_init(bar.a_empty + 8 * s, 1); }
+        for (int s = 0; s < p.v_slots; ++s) { mbar_init(bar.v_full + 8 * s, 1); mbar_init(bar.v_empty + 8 * s, 1); }
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&tm_r);
         prefetch_tensormap(&tm_v);
+        prefetch_tensormap(&tm_ahi);
+        prefetch_tensormap(&tm_alo);
         prefetch_tensormap(&tm_out);
     }
     if (warp == 1) {
@@ -198,128 +225,142 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer ---
         if (lane == 0) {
-            uint32_t it = 0;
+            uint32_t it = 0, ig = 0, ui = 0, ua = 0;   // chunks, groups, units started; A tiles requested
+            int u_a = blockIdx.x;                      // unit cursor of the A-tile requests (runs ahead)
             for (int u = blockIdx.x; u < p.units; u += gridDim.x) {
                 const Unit un = decode_unit(p, u);
                 if (*(volatile uint32_t *)&header_of(p, un.b)->full_steps == 0) {
                     if (un.rt == 0 && un.c0 == 0) header_of(p, un.b)->status = SVDCACHE_ERR_STATE;
                     continue;
                 }
-                for (int c = un.c0; c < un.c1; ++c, ++it) {
-                    const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                    if (!mbar_wait(bar.empty + 8 * s, ph ^ 1u, abort_flag)) { record_timeout(p); goto done; }
-                    const uint32_t slot = stage0 + s * p.stage_bytes;
-                    mbar_arrive_expect_tx(bar.full + 8 * s, kTileBytes + p.v_bytes);
-                    tma_load_3d(slot, &tm_r, bar.full + 8 * s, c * kTileCols, un.rt * kTileRows, un.b);
+                // request the A tiles of this unit and of the next a_bufs - 1 live units
+                while (ua < ui + (uint32_t)p.a_bufs && u_a < p.units) {
+                    const Unit ux = decode_unit(p, u_a);
+                    u_a += gridDim.x;
+                    if (*(volatile uint32_t *)&header_of(p, ux.b)->full_steps == 0) continue;
+                    const uint32_t ab = ua % p.a_bufs;
+                    if (!mbar_wait(bar.a_empty + 8 * ab, ((ua / p.a_bufs) & 1u) ^ 1u, abort_flag)) { record_timeout(p); goto done; }
+                    const uint32_t dst = a_base0 + ab * p.a_bytes;
+                    mbar_arrive_expect_tx(bar.a_full + 8 * ab, p.a_bytes);
+                    for (int kb = 0; kb < p.nkb; ++kb) {
+                        tma_load_3d(dst + kb * (kTileRows * p.kb_bytes), &tm_ahi, bar.a_full + 8 * ab,
+                                    kb * p.kb_elems, ux.rt * kTileRows, ux.b);
+                        tma_load_3d(dst + p.a_half_bytes + kb * (kTileRows * p.kb_bytes), &tm_alo, bar.a_full + 8 * ab,
+                                    kb * p.kb_elems, ux.rt * kTileRows, ux.b);
+                    }
+                    ++ua;
+                }
+                ++ui;
+                for (int cg = un.c0; cg < un.c1; cg += p.gc, ++ig) {
+                    const uint32_t vs = ig % p.v_slots;
+                    if (!mbar_wait(bar.v_empty + 8 * vs, ((ig / p.v_slots) & 1u) ^ 1u, abort_flag)) { record_timeout(p); goto done; }
+                    const uint32_t vdst = v_base0 + vs * p.vslice_bytes;
+                    mbar_arrive_expect_tx(bar.v_full + 8 * vs, p.vslice_bytes);
                     for (int kb = 0; kb < p.nkb; ++kb)
-                        tma_load_3d(slot + kTileBytes + kb * (kTileCols * p.kb_bytes), &tm_v, bar.full + 8 * s,
-                                    kb * p.kb_elems, c * kTileCols, un.b);
+                        tma_load_3d(vdst + kb * (p.gc * kTileCols * p.kb_bytes), &tm_v, bar.v_full + 8 * vs,
+                                    kb * p.kb_elems, cg * kTileCols, un.b);
+                    const int ce = min(cg + p.gc, un.c1);
+                    for (int c = cg; c < ce; ++c, ++it) {
+                        const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
+                        if (!mbar_wait(bar.empty + 8 * s, ph ^ 1u, abort_flag)) { record_timeout(p); goto done; }
+                        mbar_arrive_expect_tx(bar.full + 8 * s, kTileBytes);
+                        tma_load_3d(stage0 + s * kTileBytes, &tm_r, bar.full + 8 * s, c * kTileCols, un.rt * kTileRows, un.b);
+                    }
                 }
             }
         }
     } else if (warp == 1) {
         // -------------------------------------------------------------- MMA issuer ---
         if (lane == 0) {
-            uint32_t it = 0, ui = 0;
+            uint32_t ig = 0, ui = 0;
+            const int ksteps = p.kb_elems / 16;
             for (int u = blockIdx.x; u < p.units; u += gridDim.x) {
                 const Unit un = decode_unit(p, u);
                 if (*(volatile uint32_t *)&header_of(p, un.b)->full_steps == 0) continue;
                 const uint32_t ab = ui % p.a_bufs;
                 if (!mbar_wait(bar.a_full + 8 * ab, (ui / p.a_bufs) & 1u, abort_flag)) { record_timeout(p); goto done; }
-                tc_fence_after();
-                for (int c = un.c0; c < un.c1; ++c, ++it) {
-                    const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                    const uint32_t as = it % kAccStages, aph = (it / kAccStages) & 1u;
-                    if (!mbar_wait(bar.full + 8 * s, ph, abort_flag)) { record_timeout(p); goto done; }
-                    if (!mbar_wait(bar.acc_empty + 8 * as, aph ^ 1u, abort_flag)) { record_timeout(p); goto done; }
+                const uint64_t a_desc0 = smem_desc_kmajor(a_base0 + ab * p.a_bytes, p.kb_bytes);
+                for (int cg = un.c0; cg < un.c1; cg += p.gc, ++ig) {
+                    const uint32_t vs = ig % p.v_slots, as = ig % p.acc_stages;
+                    const int nsub = min(p.gc, un.c1 - cg);
+                    if (!mbar_wait(bar.v_full + 8 * vs, (ig / p.v_slots) & 1u, abort_flag)) { record_timeout(p); goto done; }
+                    if (!mbar_wait(bar.acc_empty + 8 * as, ((ig / p.acc_stages) & 1u) ^ 1u, abort_flag)) { record_timeout(p); goto done; }
                     tc_fence_after();
-                    issue_reconstruct_mmas(p, tmem_base + as * kTileCols, a_base0 + ab * p.a_bytes,
-                                           stage0 + s * p.stage_bytes + kTileBytes);
-                    mma_commit(bar.empty + 8 * s);
+                    const uint32_t idesc = idesc_bf16(kTileRows, nsub * kTileCols);
+                    const uint32_t d_tmem = tmem_base + as * p.acc_cols;
+                    const uint64_t v_desc0 = smem_desc_kmajor(v_base0 + vs * p.vslice_bytes, p.kb_bytes);
+                    uint32_t acc = 0;
+                    for (int part = 0; part < 2; ++part)
+                        for (int kb = 0; kb < p.nkb; ++kb) {
+                            // descriptors address in 16-byte units: add byte offsets >> 4
+                            const uint64_t a_kb = a_desc0 + ((part * p.a_half_bytes + kb * (kTileRows * p.kb_bytes)) >> 4);
+                            const uint64_t v_kb = v_desc0 + ((kb * (p.gc * kTileCols * p.kb_bytes)) >> 4);
+                            for (int ks = 0; ks < ksteps; ++ks) {
+                                mma_bf16_ss(d_tmem, a_kb + 2 * ks, v_kb + 2 * ks, idesc, acc);
+                                acc = 1;
+                            }
+                        }
+                    mma_commit(bar.v_empty + 8 * vs);
                     mma_commit(bar.acc_full + 8 * as);
                 }
                 mma_commit(bar.a_empty + 8 * ab);
                 ++ui;
             }
         }
-    } else if (warp < 6) {
-        // ---------------------------------------------------------------- epilogue ---
-        const int q = warp & 3, row = q * 32 + lane;
-        const bool leader = (warp == 2 && lane == 0);
-        uint32_t it = 0;
-        int prev_stage = -1;
-        for (int u = blockIdx.x; u < p.units; u += gridDim.x) {
-            const Unit un = decode_unit(p, u);
-            if (*(volatile uint32_t *)&header_of(p, un.b)->full_steps == 0) continue;
-            for (int c = un.c0; c < un.c1; ++c, ++it) {
-                const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                const uint32_t as = it % kAccStages, aph = (it / kAccStages) & 1u;
-                // The 128 epilogue threads meet at a named barrier every tile, so none of them
-                // may leave early: after a failed wait a thread keeps iterating with the work
-                // skipped (every later wait fails at once through the abort flag).
-                bool ok = mbar_wait(bar.acc_full + 8 * as, aph, abort_flag);
-                ok = ok && mbar_wait(bar.full + 8 * s, ph, abort_flag);
-                if (ok) {
-                    tc_fence_after();
-                    const uint32_t tile = stage0 + s * p.stage_bytes + (uint32_t)row * 128u;
-                    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + as * kTileCols;
-#pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        uint32_t acc[32];
-                        tmem_ld_32x32(taddr + half * 32, acc);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int cc = 0; cc < 4; ++cc) {
-                            const uint32_t addr = tile + (((uint32_t)(half * 4 + cc)) ^ ((uint32_t)row & 7u)) * 16u;
-                            sts128(addr, combine_chunk<false>(lds128(addr), acc + cc * 8));
-                        }
-                    }
-                    tc_fence_before();
-                    mbar_arrive(bar.acc_empty + 8 * as);
-                    fence_proxy_async();
-                } else {
-                    record_timeout(p);
-                }
-                named_barrier_sync(1, 128);
-                if (leader && ok) {
-                    tma_store_3d(&tm_out, stage0 + s * p.stage_bytes, c * kTileCols, un.rt * kTileRows, un.b);
-                    tma_store_commit();
-                    if (prev_stage >= 0) {
-                        tma_store_wait_read<1>();
-                        mbar_arrive(bar.empty + 8 * prev_stage);
-                    }
-                    prev_stage = (int)s;
-                }
-            }
-        }
-        if (leader) {
-            tma_store_wait_read<0>();
-            if (prev_stage >= 0) mbar_arrive(bar.empty + 8 * prev_stage);
-            tma_store_wait<0>();
-        }
     } else {
-        // ------------------------------------------------------------ A-operand prep ---
-        const int t = threadIdx.x - 192;
-        uint32_t ui = 0;
-        const int quads_per_row = p.k / 4;
+        // ---------------------------------------------------------------- epilogue ---
+        const int q = warp & 3, row = q * kSlabRows + lane;
+        const uint32_t grp = (uint32_t)(warp - 2) >> 2;
+        uint32_t it = 0, ig = 0;
         for (int u = blockIdx.x; u < p.units; u += gridDim.x) {
             const Unit un = decode_unit(p, u);
             if (*(volatile uint32_t *)&header_of(p, un.b)->full_steps == 0) continue;
-            const uint32_t ab = ui % p.a_bufs;
-            if (!mbar_wait(bar.a_empty + 8 * ab, ((ui / p.a_bufs) & 1u) ^ 1u, abort_flag)) { record_timeout(p); goto done; }
-            const float *chat = reinterpret_cast<const float *>(p.state + (size_t)un.b * p.state_stride + p.chat_off);
-            const uint32_t a_base = a_base0 + ab * p.a_bytes;
-            for (int idx = t; idx < kTileRows * quads_per_row; idx += 128) {
-                const int row = idx / quads_per_row, j0 = (idx - row * quads_per_row) * 4;
-                const int64_t n = (int64_t)un.rt * kTileRows + row;
-                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (n < p.N) v = *reinterpret_cast<const float4 *>(chat + n * p.k + j0);
-                store_a4(a_base, p, row, j0, v);
+            const int slab_row0 = un.rt * kTileRows + q * kSlabRows;
+            const bool slab_live = (int64_t)slab_row0 < p.N;
+            for (int cg = un.c0; cg < un.c1; cg += p.gc, ++ig) {
+                const uint32_t as = ig % p.acc_stages, aph = (ig / p.acc_stages) & 1u;
+                const int nsub = min(p.gc, un.c1 - cg);
+                for (int j = 0; j < nsub; ++j, ++it) {
+                    if ((it & 1u) != grp) continue;
+                    const int c = cg + j;
+                    const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
+                    bool ok = mbar_wait(bar.acc_full + 8 * as, aph, abort_flag);
+                    ok = ok && mbar_wait(bar.full + 8 * s, ph, abort_flag);
+                    if (!__all_sync(0xFFFFFFFFu, ok)) { record_timeout(p); goto done; }
+                    tc_fence_after();
+                    const uint32_t tile = stage0 + s * kTileBytes + (uint32_t)row * 128u;
+                    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + as * p.acc_cols + j * kTileCols;
+                    uint32_t acc0[32], acc1[32];
+                    tmem_ld_32x32(taddr, acc0);
+                    tmem_ld_32x32(taddr + 32, acc1);
+                    uint4 t[8];
+#pragma unroll
+                    for (int cc = 0; cc < 8; ++cc) t[cc] = lds128(tile + (((uint32_t)cc) ^ ((uint32_t)row & 7u)) * 16u);
+                    tmem_wait_ld();
+                    tc_fence_before();
+                    __syncwarp();
+                    // this quarter's share of the group's accumulator is in registers; the last
+                    // chunk of a short group also arrives for the chunks the group does not have
+                    if (lane == 0) mbar_arrive_n(bar.acc_empty + 8 * as, j == nsub - 1 ? 1u + (uint32_t)(p.gc - nsub) : 1u);
+#pragma unroll
+                    for (int cc = 0; cc < 8; ++cc)
+                        sts128(tile + (((uint32_t)cc) ^ ((uint32_t)row & 7u)) * 16u,
+                               combine_chunk<false>(t[cc], cc < 4 ? acc0 + cc * 8 : acc1 + (cc - 4) * 8));
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (slab_live)
+                            tma_store_3d(&tm_out, stage0 + s * kTileBytes + (uint32_t)q * kSlabBytes, c * kTileCols,
+                                         slab_row0, un.b);
+                        tma_store_commit();
+                        tma_store_wait_read<0>();
+                        mbar_arrive(bar.empty + 8 * s);
+                    }
+                    __syncwarp();
+                }
             }
-            fence_proxy_async();
-            mbar_arrive(bar.a_full + 8 * ab);
-            ++ui;
         }
+        if (lane == 0) tma_store_wait<0>();
     }
 
 done:
@@ -521,6 +562,9 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
             float *chat = reinterpret_cast<float *>(p.state + (size_t)un.b * p.state_stride + p.chat_off) + n * p.k;
             float *cout = p.C_out ? reinterpret_cast<float *>((char *)p.C_out + (size_t)un.b * p.C_stride) + n * p.k
                                   : nullptr;
+            char *st_b = p.state + (size_t)un.b * p.state_stride;
+            __nv_bfloat16 *ophi = reinterpret_cast<__nv_bfloat16 *>(st_b + p.ophi_off) + n * p.k;
+            __nv_bfloat16 *oplo = reinterpret_cast<__nv_bfloat16 *>(st_b + p.oplo_off) + n * p.k;
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + kAcc1Col;
             for (int g = 0; g * 32 < p.k; ++g) {
                 uint32_t acc[32];
@@ -543,6 +587,13 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                             }
                             *reinterpret_cast<float4 *>(chat + j) = ch;
                             if (cout) *reinterpret_cast<float4 *>(cout + j) = cv;
+                            __nv_bfloat16 h[4], l[4];
+                            split_bf16(ch.x, h[0], l[0]);
+                            split_bf16(ch.y, h[1], l[1]);
+                            split_bf16(ch.z, h[2], l[2]);
+                            split_bf16(ch.w, h[3], l[3]);
+                            *reinterpret_cast<uint2 *>(ophi + j) = *reinterpret_cast<const uint2 *>(h);
+                            *reinterpret_cast<uint2 *>(oplo + j) = *reinterpret_cast<const uint2 *>(l);
                         }
                         store_a4(a_base0, p, row, j, cv);
                     }
@@ -643,11 +694,37 @@ bool fill_params(const StepArgs &a, UmmaParams &p, int want_a_bufs) {
     if (p.stages > kMaxStages) p.stages = kMaxStages;
     p.state = (char *)a.state;
     p.state_stride = a.state_stride;
-    p.chat_off = state_layout(a.N, a.D, a.k, a.dtype).chat;
+    {
+        const StateLayout SL = state_layout(a.N, a.D, a.k, a.dtype);
+        p.chat_off = SL.chat; p.ophi_off = SL.op_hi; p.oplo_off = SL.op_lo;
+    }
     p.C_out = a.C_out;
     p.C_stride = a.C_stride;
     p.beta = a.beta;
     return true;
+}
+
+// Cached step: shared memory = A tile(s) | basis-slice ring | R ring | barriers.
+bool fill_cached(const StepArgs &a, UmmaParams &p) {
+    if (!fill_params(a, p, 1)) return false;
+    p.gc = 16384 / (kTileCols * a.k);            // basis slice (gc * 64 x k bf16) of at most 32 KB
+    if (p.gc > 4) p.gc = 4;                      // MMA N = gc * 64 <= 256
+    if (p.gc < 1) p.gc = 1;
+    p.acc_cols = p.gc * kTileCols;
+    p.acc_stages = 512 / p.acc_cols < kAccStages ? 512 / p.acc_cols : kAccStages;
+    p.vslice_bytes = (uint32_t)p.gc * kTileCols * a.k * 2;
+    p.v_slots = kMaxVSlots;
+    const size_t avail = kSmemBudget - 1024 /*alignment*/ - kBarBytes - 64;
+    const size_t fixed = (size_t)p.v_slots * p.vslice_bytes;
+    p.a_bufs = (2 * (size_t)p.a_bytes + fixed + 6 * (size_t)kTileBytes <= avail) ? 2 : 1;
+    if ((size_t)p.a_bufs * p.a_bytes + fixed + 2 * (size_t)kTileBytes > avail) return false;
+    p.stages = (int)((avail - (size_t)p.a_bufs * p.a_bytes - fixed) / kTileBytes);
+    if (p.stages > kMaxStages) p.stages = kMaxStages;
+    return true;
+}
+size_t smem_bytes_cached(const UmmaParams &p) {
+    return 1024 + (size_t)p.a_bufs * p.a_bytes + (size_t)p.v_slots * p.vslice_bytes + (size_t)p.stages * kTileBytes +
+           kBarBytes + 64;
 }
 
 size_t smem_bytes(const UmmaParams &p) {
@@ -666,40 +743,46 @@ bool shape_ok(const StepArgs &a) {
 bool umma_supported(const StepArgs &a, bool full) {
     if (!shape_ok(a)) return false;
     UmmaParams p;
-    return fill_params(a, p, full ? 1 : 2);
+    return full ? fill_params(a, p, 1) : fill_cached(a, p);
 }
 
 int umma_cached_step(const StepArgs &a, cudaStream_t s) {
     UmmaParams p{};
-    if (!fill_params(a, p, 2)) return SVDCACHE_ERR_BAD_SHAPE;
+    if (!fill_cached(a, p)) return SVDCACHE_ERR_BAD_SHAPE;
     // Split D across CTAs only when there are too few row tiles to occupy the GPU: pick the
-    // split that minimises the number of 64-column chunks the busiest CTA has to stream.
+    // split (in whole MMA groups) that minimises the chunks the busiest CTA has to stream.
     const int tiles = p.row_tiles * a.nblocks;
+    const int groups_total = (p.chunks_total + p.gc - 1) / p.gc;
     int best_load = 1 << 30;
     p.dsplit = 1;
-    for (int ds = 1; ds <= p.chunks_total && ds <= 16; ++ds) {
-        const int cps = (p.chunks_total + ds - 1) / ds;
-        const int eff = (p.chunks_total + cps - 1) / cps;
+    p.chunks_per_slice = p.chunks_total;
+    for (int ds = 1; ds <= groups_total && ds <= 16; ++ds) {
+        const int gps = (groups_total + ds - 1) / ds;            // groups per slice
+        const int eff = (groups_total + gps - 1) / gps;          // slices that result
         const int rounds = (tiles * eff + num_sms() - 1) / num_sms();
-        if (rounds * cps < best_load) { best_load = rounds * cps; p.dsplit = eff; }
+        if (rounds * gps < best_load) { best_load = rounds * gps; p.dsplit = eff; p.chunks_per_slice = gps * p.gc; }
     }
-    p.chunks_per_slice = (p.chunks_total + p.dsplit - 1) / p.dsplit;
-    p.dsplit = (p.chunks_total + p.chunks_per_slice - 1) / p.chunks_per_slice;
     p.units = tiles * p.dsplit;
 
     const StateLayout SL = state_layout(a.N, a.D, a.k, a.dtype);
     const BasisLayout BL = basis_layout(a.D, a.k, a.dtype);
-    CUtensorMap tm_r, tm_v, tm_out;
+    CUtensorMap tm_r, tm_v, tm_ahi, tm_alo, tm_out;
     int rc = make_map(&tm_r, (const char *)a.state + SL.r, a.D, a.N, a.nblocks, (uint64_t)a.D * 2, a.state_stride,
                       kTileCols, kTileRows);
     if (rc) return rc;
     rc = make_map(&tm_v, (const char *)a.basis + BL.v_bf16, a.k, a.D, a.nblocks, (uint64_t)a.k * 2, a.basis_stride,
-                  p.kb_elems, kTileCols);
+                  p.kb_elems, p.gc * kTileCols);
     if (rc) return rc;
-    rc = make_map(&tm_out, a.Fhat, a.D, a.N, a.nblocks, (uint64_t)a.ld * 2, a.Fhat_stride, kTileCols, kTileRows);
+    rc = make_map(&tm_ahi, (const char *)a.state + SL.op_hi, a.k, a.N, a.nblocks, (uint64_t)a.k * 2, a.state_stride,
+                  p.kb_elems, kTileRows);
+    if (rc) return rc;
+    rc = make_map(&tm_alo, (const char *)a.state + SL.op_lo, a.k, a.N, a.nblocks, (uint64_t)a.k * 2, a.state_stride,
+                  p.kb_elems, kTileRows);
+    if (rc) return rc;
+    rc = make_map(&tm_out, a.Fhat, a.D, a.N, a.nblocks, (uint64_t)a.ld * 2, a.Fhat_stride, kTileCols, kSlabRows);
     if (rc) return rc;
 
-    const size_t smem = smem_bytes(p);
+    const size_t smem = smem_bytes_cached(p);
     static bool attr_set = false;
     if (!attr_set) {
         rc = record_cuda(cudaFuncSetAttribute(umma_cached_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -708,7 +791,7 @@ int umma_cached_step(const StepArgs &a, cudaStream_t s) {
         attr_set = true;
     }
     const int grid = p.units < num_sms() ? p.units : num_sms();
-    umma_cached_kernel<<<grid, kThreadsUmma, smem, s>>>(tm_r, tm_v, tm_out, p);
+    umma_cached_kernel<<<grid, kThreadsCached, smem, s>>>(tm_r, tm_v, tm_ahi, tm_alo, tm_out, p);
     count_launch();
     return check_last_launch();
 }
