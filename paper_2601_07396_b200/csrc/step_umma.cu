@@ -20,7 +20,6 @@ using namespace sm100;
 
 namespace {
 
-constexpr int kThreadsUmma = 320;
 constexpr int kTileRows = 128;      // MMA M
 constexpr int kTileCols = 64;       // columns of D per stage (MMA N in the reconstruct GEMM)
 constexpr int kTileBytes = kTileRows * kTileCols * 2;   // 16 KB
@@ -35,9 +34,11 @@ struct UmmaParams {
     int row_tiles, chunks_total, dsplit, chunks_per_slice, units;
     int kb_elems, kb_bytes, nkb;         // K-block of the rank dimension: min(k, 64) elements
     int stages, a_bufs;
-    uint32_t a_half_bytes, a_bytes, v_bytes, stage_bytes;
-    int gc, acc_stages, acc_cols, v_slots;   // cached step: chunks per MMA group, TMEM ring, basis ring
+    uint32_t a_half_bytes, a_bytes;
+    int gc, acc_stages, acc_cols, v_slots;   // chunks per MMA group, TMEM ring, basis ring
     uint32_t vslice_bytes;
+    int nacc;                                // full step: pass-1 accumulators
+    uint32_t a_region_bytes, chat_stage_off; // full step: A operand (+ Chat staging when k < 64)
     char *state;
     size_t state_stride, chat_off, ophi_off, oplo_off;
     float *C_out;
@@ -123,42 +124,6 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
 }
 __device__ __forceinline__ void sts64(uint32_t addr, uint32_t x, uint32_t y) {
     asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(addr), "r"(x), "r"(y) : "memory");
-}
-
-// Write 4 consecutive coefficients (columns j0..j0+3 of tile row `row`) into the A operand:
-// a K-major, swizzled tile made of K-blocks of kb_elems columns, stored twice -- the bf16
-// rounding of each value ("hi") and the bf16 rounding of what that rounding lost ("lo").
-// hi + lo carries ~16 mantissa bits, so the product with V_k is good to ~1e-5 relative.
-__device__ __forceinline__ void store_a4(uint32_t a_base, const UmmaParams &p, int row, int j0, float4 v) {
-    const int kb = j0 / p.kb_elems, jj = j0 - kb * p.kb_elems;
-    const uint32_t chunk = (uint32_t)jj >> 3, within = ((uint32_t)jj & 7u) * 2u;
-    const uint32_t addr = a_base + (uint32_t)kb * (kTileRows * p.kb_bytes) + (uint32_t)row * p.kb_bytes +
-                          swizzled_chunk((uint32_t)row, chunk, (uint32_t)p.kb_bytes) * 16u + within;
-    const __nv_bfloat162 h01 = __floats2bfloat162_rn(v.x, v.y), h23 = __floats2bfloat162_rn(v.z, v.w);
-    const float2 f01 = __bfloat1622float2(h01), f23 = __bfloat1622float2(h23);
-    const __nv_bfloat162 l01 = __floats2bfloat162_rn(v.x - f01.x, v.y - f01.y);
-    const __nv_bfloat162 l23 = __floats2bfloat162_rn(v.z - f23.x, v.w - f23.y);
-    sts64(addr, *reinterpret_cast<const uint32_t *>(&h01), *reinterpret_cast<const uint32_t *>(&h23));
-    sts64(addr + p.a_half_bytes, *reinterpret_cast<const uint32_t *>(&l01), *reinterpret_cast<const uint32_t *>(&l23));
-}
-
-// issue the 2 * k/16 MMAs of one 128 x 64 output tile: D = (A_hi + A_lo)[128 x k] * B[64 x k]^T
-__device__ __forceinline__ void issue_reconstruct_mmas(const UmmaParams &p, uint32_t d_tmem, uint32_t a_base,
-                                                       uint32_t v_base) {
-    const uint32_t idesc = idesc_bf16(kTileRows, kTileCols);
-    const int ksteps = p.kb_elems / 16;
-    bool acc = false;
-    for (int part = 0; part < 2; ++part) {
-        for (int kb = 0; kb < p.nkb; ++kb) {
-            const uint32_t a_kb = a_base + (uint32_t)part * p.a_half_bytes + (uint32_t)kb * (kTileRows * p.kb_bytes);
-            const uint32_t v_kb = v_base + (uint32_t)kb * (kTileCols * p.kb_bytes);
-            for (int ks = 0; ks < ksteps; ++ks) {
-                mma_bf16_ss(d_tmem, smem_desc_kmajor(a_kb + ks * 32, p.kb_bytes),
-                            smem_desc_kmajor(v_kb + ks * 32, p.kb_bytes), idesc, acc ? 1u : 0u);
-                acc = true;
-            }
-        }
-    }
 }
 
 // ======================================================================================
@@ -375,24 +340,71 @@ done:
 // ======================================================================================
 // Full step (Eq. 8 - Eq. 11):  C = F V_k,  Chat <- EMA(C),  R = F - C V_k^T
 //
-// A unit is one 128-row tile of one block.  Pass 1 streams the tile's F in 64-column
-// slices and accumulates C (128 x k, fp32) in TMEM: A = F slice, B = matching slice of
-// V_k^T.  The C warps then read C from TMEM, apply the EMA to the state, and write C as a
-// split-bf16 A operand.  Pass 2 streams the same F slices again (in reverse order, so the
-// most recently touched ones come first and are still in L2) with slices of V_k, forms
-// C V_k^T per slice in TMEM, and the epilogue stores R = F - C V_k^T through TMA.
+// A unit is one 128-row tile of one block.
+//   Pass 1 streams the tile's F in 64-column chunks and accumulates C (128 x k, fp32) in
+//     TMEM: A = F chunk, B = matching columns of V_k^T.  Consecutive chunks go to different
+//     accumulators (up to four), so their dependent MMA chains overlap; the C warps add them.
+//   The C warps read C from TMEM, apply the EMA against the previous Chat (staged by TMA in
+//     the A-operand region and converted in place), write Chat, and leave C as a split-bf16
+//     A operand in shared memory -- which also goes out, as it is, as the state's operand copy.
+//   Pass 2 streams the same F chunks again, last group first (the most recently read ones
+//     are the likeliest to sit in L2), with V_k slices of gc*64 rows: C V_k^T per group in
+//     TMEM, and the epilogue stores R = F - C V_k^T through TMA.
+// The pass-1 accumulators overlay the pass-2 accumulator ring, so pass 1 of a unit starts
+// once the epilogue has drained the previous unit.
+//
+// Warp roles (448 threads): 0 = TMA producer, 1 = MMA issuer (+ TMEM owner), 2..9 = two
+// epilogue groups of four warps, 10..13 = C warps.
 // ======================================================================================
-constexpr uint32_t kAcc1Col = kAccStages * kTileCols;   // C accumulator sits after the pass-2 ring
+constexpr int kThreadsFull = 448;
+constexpr uint32_t kBlk32Bytes = kTileRows * 128u;   // 16 KB: 128 rows x 32 fp32 (or x 64 bf16)
 
-__global__ void __launch_bounds__(kThreadsUmma, 1)
+// 32 consecutive coefficients of one row: EMA against `prev`, global stores, split-bf16 pack.
+struct RowOut {
+    float *chat, *cout;          // global rows (nullptr: do not store)
+};
+
+__device__ __forceinline__ void load_row32(uint32_t row_addr, uint32_t row, uint32_t row_bytes, int ncols, float (&v)[32]) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        if (i * 4 < ncols) {
+            const uint4 t = lds128(row_addr + swizzled_chunk(row, (uint32_t)i, row_bytes) * 16u);
+            v[4 * i] = __uint_as_float(t.x); v[4 * i + 1] = __uint_as_float(t.y);
+            v[4 * i + 2] = __uint_as_float(t.z); v[4 * i + 3] = __uint_as_float(t.w);
+        }
+    }
+}
+
+// hi/lo bf16 of 8 consecutive values -> one 16-byte chunk each
+__device__ __forceinline__ void pack_split8(const float *v, uint4 &hi, uint4 &lo) {
+    uint32_t h[4], l[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const __nv_bfloat162 hh = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+        const float2 hf = __bfloat1622float2(hh);
+        const __nv_bfloat162 ll = __floats2bfloat162_rn(v[2 * i] - hf.x, v[2 * i + 1] - hf.y);
+        h[i] = *reinterpret_cast<const uint32_t *>(&hh);
+        l[i] = *reinterpret_cast<const uint32_t *>(&ll);
+    }
+    hi = make_uint4(h[0], h[1], h[2], h[3]);
+    lo = make_uint4(l[0], l[1], l[2], l[3]);
+}
+
+__global__ void __launch_bounds__(kThreadsFull, 1)
 umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant__ CUtensorMap tm_vt,
                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_rout,
-                 const UmmaParams p) {
+                 const __grid_constant__ CUtensorMap tm_chat, const UmmaParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t a_base0 = base;
-    const uint32_t stage0 = a_base0 + p.a_bytes;
-    const Bars bar = bars_at(stage0 + (uint32_t)p.stages * p.stage_bytes);
+    const uint32_t a_base = base;                                     // A operand (and, for k >= 64, staged Chat)
+    const uint32_t chat_base = a_base + p.chat_stage_off;             // == a_base when k >= 64
+    const uint32_t v_base0 = a_base + p.a_region_bytes;
+    const uint32_t stage0 = v_base0 + (uint32_t)p.v_slots * p.vslice_bytes;
+    const Bars bar = bars_at(stage0 + (uint32_t)p.stages * kTileBytes);
+    // barriers beyond the ring ones: c_full (C accumulated), a_full (A operand written),
+    // p2_done (pass-2 MMAs of the unit finished: the A region may be restaged), chat_full
+    // (previous Chat staged)
+    const uint32_t chat_full = bar.a_full + 8, p2_done = bar.c_done;
     uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
     volatile int *abort_flag = reinterpret_cast<volatile int *>(gen_base + (bar.abort_flag - base));
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(gen_base + (bar.tmem_slot - base));
@@ -400,18 +412,25 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t tmem_cols = 512;
     const int CT = p.chunks_total;
+    const int G = (CT + p.gc - 1) / p.gc;               // groups per pass
+    const uint32_t a_part = p.k >= 64 ? kBlk32Bytes : p.a_half_bytes;   // hi -> lo distance
+    const uint32_t a_kb = 2u * kBlk32Bytes;                             // K-block distance (k >= 64)
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < p.stages; ++s) { mbar_init(bar.full + 8 * s, 1); mbar_init(bar.empty + 8 * s, 2); }
-        for (int s = 0; s < kAccStages; ++s) { mbar_init(bar.acc_full + 8 * s, 1); mbar_init(bar.acc_empty + 8 * s, 128); }
+        for (int s = 0; s < p.stages; ++s) { mbar_init(bar.full + 8 * s, 1); mbar_init(bar.empty + 8 * s, 4); }
+        for (int s = 0; s < p.acc_stages; ++s) { mbar_init(bar.acc_full + 8 * s, 1); mbar_init(bar.acc_empty + 8 * s, 4 * p.gc); }
+        for (int s = 0; s < p.v_slots; ++s) { mbar_init(bar.v_full + 8 * s, 1); mbar_init(bar.v_empty + 8 * s, 1); }
         mbar_init(bar.a_full, 128);
+        mbar_init(chat_full, 1);
         mbar_init(bar.c_full, 1);
+        mbar_init(p2_done, 1);
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&tm_f);
         prefetch_tensormap(&tm_vt);
         prefetch_tensormap(&tm_v);
         prefetch_tensormap(&tm_rout);
+        prefetch_tensormap(&tm_chat);
     }
     if (warp == 1) {
         tmem_alloc(bar.tmem_slot, tmem_cols);
@@ -425,191 +444,297 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer ---
         if (lane == 0) {
-            uint32_t it = 0;
+            const uint64_t pol_keep = policy_evict_last(), pol_drop = policy_evict_first();
+            uint32_t it = 0, iv = 0;   // F chunks, basis slices requested so far
             for (int u = blockIdx.x; u < p.units; u += gridDim.x) {
                 const Unit un = decode_unit(p, u);
-                for (int c = 0; c < CT; ++c, ++it) {            // pass 1: F slice + V^T slice
-                    const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                    if (!mbar_wait(bar.empty + 8 * s, ph ^ 1u, abort_flag)) { record_timeout(p); goto done; }
-                    const uint32_t slot = stage0 + s * p.stage_bytes;
-                    mbar_arrive_expect_tx(bar.full + 8 * s, kTileBytes + (uint32_t)p.k * 128u);
-                    tma_load_3d(slot, &tm_f, bar.full + 8 * s, c * kTileCols, un.rt * kTileRows, un.b);
-                    tma_load_3d(slot + kTileBytes, &tm_vt, bar.full + 8 * s, c * kTileCols, 0, un.b);
-                }
-                for (int c2 = 0; c2 < CT; ++c2, ++it) {         // pass 2: F slice again + V slice
-                    const int c = CT - 1 - c2;
-                    const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                    if (!mbar_wait(bar.empty + 8 * s, ph ^ 1u, abort_flag)) { record_timeout(p); goto done; }
-                    const uint32_t slot = stage0 + s * p.stage_bytes;
-                    mbar_arrive_expect_tx(bar.full + 8 * s, kTileBytes + p.v_bytes);
-                    tma_load_3d(slot, &tm_f, bar.full + 8 * s, c * kTileCols, un.rt * kTileRows, un.b);
-                    for (int kb = 0; kb < p.nkb; ++kb)
-                        tma_load_3d(slot + kTileBytes + kb * (kTileCols * p.kb_bytes), &tm_v, bar.full + 8 * s,
-                                    kb * p.kb_elems, c * kTileCols, un.b);
+                for (int pass = 0; pass < 2; ++pass) {
+                    for (int g = 0; g < G; ++g, ++iv) {
+                        const int cg = (pass == 0 ? g : G - 1 - g) * p.gc;
+                        const int ce = min(cg + p.gc, CT);
+                        const uint32_t vs = iv % p.v_slots;
+                        if (!mbar_wait(bar.v_empty + 8 * vs, ((iv / p.v_slots) & 1u) ^ 1u, abort_flag)) { record_timeout(p); goto done; }
+                        const uint32_t vdst = v_base0 + vs * p.vslice_bytes;
+                        mbar_arrive_expect_tx(bar.v_full + 8 * vs, p.vslice_bytes);
+                        if (pass == 0) {   // V_k^T columns of each chunk: gc boxes of k rows x 64
+                            for (int j = 0; j < p.gc; ++j)
+                                tma_load_3d(vdst + j * (p.k * 128), &tm_vt, bar.v_full + 8 * vs, (cg + j) * kTileCols, 0, un.b);
+                        } else {           // V_k rows of the group: one box of gc*64 rows per K block
+                            for (int kb = 0; kb < p.nkb; ++kb)
+                                tma_load_3d(vdst + kb * (p.gc * kTileCols * p.kb_bytes), &tm_v, bar.v_full + 8 * vs,
+                                            kb * p.kb_elems, cg * kTileCols, un.b);
+                        }
+                        for (int c = cg; c < ce; ++c, ++it) {
+                            const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
+                            if (!mbar_wait(bar.empty + 8 * s, ph ^ 1u, abort_flag)) { record_timeout(p); goto done; }
+                            mbar_arrive_expect_tx(bar.full + 8 * s, kTileBytes);
+                            tma_load_3d_hint(stage0 + s * kTileBytes, &tm_f, bar.full + 8 * s, c * kTileCols,
+                                             un.rt * kTileRows, un.b, pass == 0 ? pol_keep : pol_drop);
+                        }
+                    }
                 }
             }
         }
     } else if (warp == 1) {
         // -------------------------------------------------------------- MMA issuer ---
         if (lane == 0) {
-            uint32_t it = 0, ia = 0, ui = 0;
+            uint32_t it = 0, iv = 0, ig = 0, ui = 0;   // F chunks, basis slices, pass-2 groups, units
             const uint32_t idesc1 = idesc_bf16(kTileRows, p.k);
+            const int ksteps = p.kb_elems / 16;
+            const uint64_t a_desc0 = smem_desc_kmajor(a_base, p.kb_bytes);
             for (int u = blockIdx.x; u < p.units; u += gridDim.x, ++ui) {
-                for (int c = 0; c < CT; ++c, ++it) {            // pass 1: C += F_slice * (V^T slice)^T
-                    const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                    if (!mbar_wait(bar.full + 8 * s, ph, abort_flag)) { record_timeout(p); goto done; }
-                    tc_fence_after();
-                    const uint32_t slot = stage0 + s * p.stage_bytes;
+                // the pass-1 accumulators overlay the pass-2 ring: wait until it has drained
+                for (int as = 0; as < p.acc_stages; ++as) {
+                    const uint32_t uses = (ig + p.acc_stages - 1 - as) / p.acc_stages;   // uses of stage `as` so far
+                    if (!mbar_wait(bar.acc_empty + 8 * as, (uses & 1u) ^ 1u, abort_flag)) { record_timeout(p); goto done; }
+                }
+                tc_fence_after();
+                for (int g = 0; g < G; ++g, ++iv) {                 // pass 1: C_a += F_chunk (V^T chunk)^T
+                    const int cg = g * p.gc, ce = min(cg + p.gc, CT);
+                    const uint32_t vs = iv % p.v_slots;
+                    if (!mbar_wait(bar.v_full + 8 * vs, (iv / p.v_slots) & 1u, abort_flag)) { record_timeout(p); goto done; }
+                    for (int c = cg; c < ce; ++c, ++it) {
+                        const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
+                        if (!mbar_wait(bar.full + 8 * s, ph, abort_flag)) { record_timeout(p); goto done; }
+                        tc_fence_after();
+                        const uint64_t fd = smem_desc_kmajor(stage0 + s * kTileBytes, 128);
+                        const uint64_t vd = smem_desc_kmajor(v_base0 + vs * p.vslice_bytes + (c - cg) * (p.k * 128), 128);
+                        const uint32_t d = tmem_base + (uint32_t)(c % p.nacc) * p.k;
 #pragma unroll
-                    for (int ks = 0; ks < kTileCols / 16; ++ks)
-                        mma_bf16_ss(tmem_base + kAcc1Col, smem_desc_kmajor(slot + ks * 32, 128),
-                                    smem_desc_kmajor(slot + kTileBytes + ks * 32, 128), idesc1,
-                                    (c | ks) != 0 ? 1u : 0u);
-                    mma_commit(bar.empty + 8 * s);
-                    mbar_arrive(bar.empty + 8 * s);   // the F slice is not stored in pass 1: second arrival
+                        for (int ks = 0; ks < kTileCols / 16; ++ks)
+                            mma_bf16_ss(d, fd + 2 * ks, vd + 2 * ks, idesc1, (c >= p.nacc || ks > 0) ? 1u : 0u);
+                        mma_commit(bar.empty + 8 * s);
+                        mbar_arrive_n(bar.empty + 8 * s, 3);   // pass 1 has no slab stores: their three other arrivals
+                    }
+                    mma_commit(bar.v_empty + 8 * vs);
                 }
                 mma_commit(bar.c_full);
                 if (!mbar_wait(bar.a_full, ui & 1u, abort_flag)) { record_timeout(p); goto done; }
                 tc_fence_after();
-                for (int c2 = 0; c2 < CT; ++c2, ++it, ++ia) {   // pass 2: acc = C * (V slice)^T
-                    const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                    const uint32_t as = ia % kAccStages, aph = (ia / kAccStages) & 1u;
-                    if (!mbar_wait(bar.full + 8 * s, ph, abort_flag)) { record_timeout(p); goto done; }
-                    if (!mbar_wait(bar.acc_empty + 8 * as, aph ^ 1u, abort_flag)) { record_timeout(p); goto done; }
+                for (int g = 0; g < G; ++g, ++iv, ++ig) {           // pass 2: acc = C (V slice)^T
+                    const int cg = (G - 1 - g) * p.gc;
+                    const int nsub = min(p.gc, CT - cg);
+                    const uint32_t vs = iv % p.v_slots, as = ig % p.acc_stages;
+                    if (!mbar_wait(bar.v_full + 8 * vs, (iv / p.v_slots) & 1u, abort_flag)) { record_timeout(p); goto done; }
+                    if (!mbar_wait(bar.acc_empty + 8 * as, ((ig / p.acc_stages) & 1u) ^ 1u, abort_flag)) { record_timeout(p); goto done; }
                     tc_fence_after();
-                    issue_reconstruct_mmas(p, tmem_base + as * kTileCols, a_base0,
-                                           stage0 + s * p.stage_bytes + kTileBytes);
-                    mma_commit(bar.empty + 8 * s);
+                    const uint32_t idesc = idesc_bf16(kTileRows, nsub * kTileCols);
+                    const uint32_t d_tmem = tmem_base + as * p.acc_cols;
+                    const uint64_t v_desc0 = smem_desc_kmajor(v_base0 + vs * p.vslice_bytes, p.kb_bytes);
+                    uint32_t acc = 0;
+                    for (int part = 0; part < 2; ++part)
+                        for (int kb = 0; kb < p.nkb; ++kb) {
+                            const uint64_t ad = a_desc0 + ((part * a_part + kb * a_kb) >> 4);
+                            const uint64_t vd = v_desc0 + ((kb * (p.gc * kTileCols * p.kb_bytes)) >> 4);
+                            for (int ks = 0; ks < ksteps; ++ks) {
+                                mma_bf16_ss(d_tmem, ad + 2 * ks, vd + 2 * ks, idesc, acc);
+                                acc = 1;
+                            }
+                        }
+                    mma_commit(bar.v_empty + 8 * vs);
                     mma_commit(bar.acc_full + 8 * as);
                 }
+                mma_commit(p2_done);
+                it += CT;   // pass-2 slots are consumed by the epilogue alone
             }
         }
-    } else if (warp < 6) {
+    } else if (warp < 10) {
         // ------------------------------------------- epilogue: R = F - C V_k^T, TMA store ---
-        const int q = warp & 3, row = q * 32 + lane;
-        const bool leader = (warp == 2 && lane == 0);
-        uint32_t it = 0, ia = 0;
-        int prev_stage = -1;
+        const int q = warp & 3, row = q * kSlabRows + lane;
+        const uint32_t grp = (uint32_t)(warp - 2) >> 2;
+        uint32_t it = 0, ig = 0;
         for (int u = blockIdx.x; u < p.units; u += gridDim.x) {
             const Unit un = decode_unit(p, u);
-            it += CT;   // pass 1 stages are consumed by the MMA warp alone
-            for (int c2 = 0; c2 < CT; ++c2, ++it, ++ia) {
-                const int c = CT - 1 - c2;
-                const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                const uint32_t as = ia % kAccStages, aph = (ia / kAccStages) & 1u;
-                bool ok = mbar_wait(bar.acc_full + 8 * as, aph, abort_flag);
-                ok = ok && mbar_wait(bar.full + 8 * s, ph, abort_flag);
-                if (ok) {
+            const int slab_row0 = un.rt * kTileRows + q * kSlabRows;
+            const bool slab_live = (int64_t)slab_row0 < p.N;
+            it += CT;   // pass-1 slots are consumed by the MMA warp alone
+            for (int g = 0; g < G; ++g, ++ig) {
+                const int cg = (G - 1 - g) * p.gc;
+                const int nsub = min(p.gc, CT - cg);
+                const uint32_t as = ig % p.acc_stages, aph = (ig / p.acc_stages) & 1u;
+                for (int j = 0; j < nsub; ++j, ++it) {
+                    if ((it & 1u) != grp) continue;
+                    const int c = cg + j;
+                    const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
+                    bool ok = mbar_wait(bar.acc_full + 8 * as, aph, abort_flag);
+                    ok = ok && mbar_wait(bar.full + 8 * s, ph, abort_flag);
+                    if (!__all_sync(0xFFFFFFFFu, ok)) { record_timeout(p); goto done; }
                     tc_fence_after();
-                    const uint32_t tile = stage0 + s * p.stage_bytes + (uint32_t)row * 128u;
-                    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + as * kTileCols;
+                    const uint32_t tile = stage0 + s * kTileBytes + (uint32_t)row * 128u;
+                    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + as * p.acc_cols + j * kTileCols;
+                    uint32_t acc0[32], acc1[32];
+                    tmem_ld_32x32(taddr, acc0);
+                    tmem_ld_32x32(taddr + 32, acc1);
+                    uint4 t[8];
 #pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        uint32_t acc[32];
-                        tmem_ld_32x32(taddr + half * 32, acc);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int cc = 0; cc < 4; ++cc) {
-                            const uint32_t addr = tile + (((uint32_t)(half * 4 + cc)) ^ ((uint32_t)row & 7u)) * 16u;
-                            sts128(addr, combine_chunk<true>(lds128(addr), acc + cc * 8));
-                        }
-                    }
+                    for (int cc = 0; cc < 8; ++cc) t[cc] = lds128(tile + (((uint32_t)cc) ^ ((uint32_t)row & 7u)) * 16u);
+                    tmem_wait_ld();
                     tc_fence_before();
-                    mbar_arrive(bar.acc_empty + 8 * as);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_n(bar.acc_empty + 8 * as, j == nsub - 1 ? 1u + (uint32_t)(p.gc - nsub) : 1u);
+#pragma unroll
+                    for (int cc = 0; cc < 8; ++cc)
+                        sts128(tile + (((uint32_t)cc) ^ ((uint32_t)row & 7u)) * 16u,
+                               combine_chunk<true>(t[cc], cc < 4 ? acc0 + cc * 8 : acc1 + (cc - 4) * 8));
                     fence_proxy_async();
-                } else {
-                    record_timeout(p);
-                }
-                named_barrier_sync(1, 128);
-                if (leader && ok) {
-                    tma_store_3d(&tm_rout, stage0 + s * p.stage_bytes, c * kTileCols, un.rt * kTileRows, un.b);
-                    tma_store_commit();
-                    // A stage goes back to the producer once its store has read it.  Inside a
-                    // unit that is checked one tile late; the unit's last tile is released at
-                    // once, because the next unit's pass 1 needs the whole ring to get going.
-                    if (c2 == CT - 1) {
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (slab_live)
+                            tma_store_3d(&tm_rout, stage0 + s * kTileBytes + (uint32_t)q * kSlabBytes, c * kTileCols,
+                                         slab_row0, un.b);
+                        tma_store_commit();
                         tma_store_wait_read<0>();
-                        if (prev_stage >= 0) mbar_arrive(bar.empty + 8 * prev_stage);
                         mbar_arrive(bar.empty + 8 * s);
-                        prev_stage = -1;
-                    } else {
-                        if (prev_stage >= 0) {
-                            tma_store_wait_read<1>();
-                            mbar_arrive(bar.empty + 8 * prev_stage);
-                        }
-                        prev_stage = (int)s;
                     }
+                    __syncwarp();
                 }
             }
         }
-        if (leader) {
-            tma_store_wait_read<0>();
-            if (prev_stage >= 0) mbar_arrive(bar.empty + 8 * prev_stage);
-            tma_store_wait<0>();
-        }
+        if (lane == 0) tma_store_wait<0>();
     } else {
-        // --------------------------- C warps: TMEM -> EMA on the state -> split-bf16 A operand ---
+        // ------------- C warps: TMEM -> EMA -> Chat, split-bf16 A operand (+ its copy in the state) ---
         const int q = warp & 3, row = q * 32 + lane;
         const float beta = p.beta, omb = 1.0f - p.beta;
-        uint32_t ui = 0;
+        const bool issuer = (warp == 10 && lane == 0);
+        const uint32_t chat_row_bytes = p.k >= 32 ? 128u : (uint32_t)p.k * 4u;
+        const int nblk = (p.k + 31) / 32;
+        const int nacc_used = CT < p.nacc ? CT : p.nacc;
+        uint32_t ui = 0, nchat = 0;   // units done; Chat tiles consumed
+        bool alive = true;
+
+        auto request_chat = [&](const Unit &x) {   // previous Chat of unit x -> staging, by TMA
+            mbar_arrive_expect_tx(chat_full, (uint32_t)kTileRows * p.k * 4u);
+            for (int b = 0; b < nblk; ++b)
+                tma_load_3d(chat_base + b * kBlk32Bytes, &tm_chat, chat_full, b * 32, x.rt * kTileRows, x.b);
+        };
+        if (issuer && (int)blockIdx.x < p.units) {
+            const Unit x = decode_unit(p, blockIdx.x);
+            if (*(volatile uint32_t *)&header_of(p, x.b)->full_steps != 0) request_chat(x);
+        }
         for (int u = blockIdx.x; u < p.units; u += gridDim.x, ++ui) {
             const Unit un = decode_unit(p, u);
             StateHeader *hdr = header_of(p, un.b);
             const bool first = *(volatile uint32_t *)&hdr->full_steps == 0;
-            if (!mbar_wait(bar.c_full, ui & 1u, abort_flag)) { record_timeout(p); goto done; }
-            tc_fence_after();
-            const int64_t n = (int64_t)un.rt * kTileRows + row;
-            float *chat = reinterpret_cast<float *>(p.state + (size_t)un.b * p.state_stride + p.chat_off) + n * p.k;
-            float *cout = p.C_out ? reinterpret_cast<float *>((char *)p.C_out + (size_t)un.b * p.C_stride) + n * p.k
-                                  : nullptr;
-            char *st_b = p.state + (size_t)un.b * p.state_stride;
-            __nv_bfloat16 *ophi = reinterpret_cast<__nv_bfloat16 *>(st_b + p.ophi_off) + n * p.k;
-            __nv_bfloat16 *oplo = reinterpret_cast<__nv_bfloat16 *>(st_b + p.oplo_off) + n * p.k;
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + kAcc1Col;
-            for (int g = 0; g * 32 < p.k; ++g) {
-                uint32_t acc[32];
-                tmem_ld_32x32(taddr + g * 32, acc);
-                tmem_wait_ld();
+            if (alive && !first) {
+                alive = __all_sync(0xFFFFFFFFu, mbar_wait(chat_full, nchat & 1u, abort_flag));
+                ++nchat;
+            }
+            if (alive) alive = __all_sync(0xFFFFFFFFu, mbar_wait(bar.c_full, ui & 1u, abort_flag));
+            if (alive) {
+                tc_fence_after();
+                const int64_t n = (int64_t)un.rt * kTileRows + row;
+                const bool row_live = n < p.N;
+                char *st_b = p.state + (size_t)un.b * p.state_stride;
+                float *chat_g = reinterpret_cast<float *>(st_b + p.chat_off) + n * p.k;
+                float *cout_g = p.C_out ? reinterpret_cast<float *>((char *)p.C_out + (size_t)un.b * p.C_stride) + n * p.k
+                                        : nullptr;
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+                const int nkb64 = p.k >= 64 ? p.nkb : 1;
+                for (int kb = 0; kb < nkb64; ++kb) {
+                    // staged previous Chat of this row: the block holding columns kb*64 .. +31 (A) and
+                    // the one holding +32 .. +63 (B).  For k >= 64 they are exactly where this row's
+                    // hi and lo operand rows go, so B is read before anything is written.
+                    const uint32_t stA = chat_base + (uint32_t)(2 * kb) * kBlk32Bytes + (uint32_t)row * chat_row_bytes;
+                    const uint32_t stB = stA + kBlk32Bytes;
+                    const uint32_t hi_row = a_base + (uint32_t)kb * a_kb + (uint32_t)row * p.kb_bytes;
+                    const uint32_t lo_row = hi_row + a_part;
+                    const int halves = p.k >= 64 ? 2 : 1;
+                    float prevB[32];
+                    if (!first && halves == 2) load_row32(stB, (uint32_t)row, chat_row_bytes, 32, prevB);
+                    for (int h = 0; h < halves; ++h) {
+                        const int col0 = kb * 64 + h * 32;
+                        const int ncols = p.k - col0 < 32 ? p.k - col0 : 32;
+                        float cs[32];
+                        {
+                            uint32_t tmp[32];
+                            tmem_ld_32x32(taddr + col0, tmp);
+                            tmem_wait_ld();
 #pragma unroll
-                for (int j4 = 0; j4 < 8; ++j4) {
-                    const int j = g * 32 + j4 * 4;
-                    if (j < p.k) {
-                        const float4 cv = make_float4(__uint_as_float(acc[j4 * 4]), __uint_as_float(acc[j4 * 4 + 1]),
-                                                      __uint_as_float(acc[j4 * 4 + 2]), __uint_as_float(acc[j4 * 4 + 3]));
-                        if (n < p.N) {
-                            float4 ch = cv;
-                            if (!first) {
-                                const float4 pv = *reinterpret_cast<const float4 *>(chat + j);
-                                ch.x = fmaf(beta, pv.x, omb * cv.x);
-                                ch.y = fmaf(beta, pv.y, omb * cv.y);
-                                ch.z = fmaf(beta, pv.z, omb * cv.z);
-                                ch.w = fmaf(beta, pv.w, omb * cv.w);
+                            for (int i = 0; i < 32; ++i) cs[i] = __uint_as_float(tmp[i]);
+                            for (int a = 1; a < nacc_used; ++a) {
+                                tmem_ld_32x32(taddr + a * p.k + col0, tmp);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) cs[i] += __uint_as_float(tmp[i]);
                             }
-                            *reinterpret_cast<float4 *>(chat + j) = ch;
-                            if (cout) *reinterpret_cast<float4 *>(cout + j) = cv;
-                            __nv_bfloat16 h[4], l[4];
-                            split_bf16(ch.x, h[0], l[0]);
-                            split_bf16(ch.y, h[1], l[1]);
-                            split_bf16(ch.z, h[2], l[2]);
-                            split_bf16(ch.w, h[3], l[3]);
-                            *reinterpret_cast<uint2 *>(ophi + j) = *reinterpret_cast<const uint2 *>(h);
-                            *reinterpret_cast<uint2 *>(oplo + j) = *reinterpret_cast<const uint2 *>(l);
                         }
-                        store_a4(a_base0, p, row, j, cv);
+                        float ch[32];
+                        if (first) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) ch[i] = cs[i];
+                        } else {
+                            if (h == 0) load_row32(stA, (uint32_t)row, chat_row_bytes, ncols, ch);
+                            else {
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) ch[i] = prevB[i];
+                            }
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) ch[i] = fmaf(beta, ch[i], omb * cs[i]);
+                        }
+                        if (row_live) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                if (i * 4 < ncols) {
+                                    *reinterpret_cast<float4 *>(chat_g + col0 + 4 * i) =
+                                        make_float4(ch[4 * i], ch[4 * i + 1], ch[4 * i + 2], ch[4 * i + 3]);
+                                    if (cout_g)
+                                        *reinterpret_cast<float4 *>(cout_g + col0 + 4 * i) =
+                                            make_float4(cs[4 * i], cs[4 * i + 1], cs[4 * i + 2], cs[4 * i + 3]);
+                                }
+                            }
+                        }
+                        // split-bf16 operand of C (not of Chat) for pass 2 ...
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            if (i * 8 < ncols) {
+                                uint4 hi, lo;
+                                pack_split8(cs + 8 * i, hi, lo);
+                                const uint32_t chunk = swizzled_chunk((uint32_t)row, (uint32_t)(h * 4 + i), (uint32_t)p.kb_bytes) * 16u;
+                                sts128(hi_row + chunk, hi);
+                                sts128(lo_row + chunk, lo);
+                            }
+                        }
+                        // ... while the state keeps the split of the new Chat
+                        if (row_live) {
+                            __nv_bfloat16 *ohi = reinterpret_cast<__nv_bfloat16 *>(st_b + p.ophi_off) + n * p.k + col0;
+                            __nv_bfloat16 *olo = reinterpret_cast<__nv_bfloat16 *>(st_b + p.oplo_off) + n * p.k + col0;
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                if (i * 8 < ncols) {
+                                    uint4 hi, lo;
+                                    pack_split8(ch + 8 * i, hi, lo);
+                                    *reinterpret_cast<uint4 *>(ohi + 8 * i) = hi;
+                                    *reinterpret_cast<uint4 *>(olo + 8 * i) = lo;
+                                }
+                            }
+                        }
                     }
                 }
+                tc_fence_before();
+                fence_proxy_async();
+                mbar_arrive(bar.a_full);
+                // count this unit; the last unit of a block to get here counts the full step
+                if (issuer) {
+                    const uint32_t prev = atomicAdd(&hdr->done, 1u);
+                    if (prev == (uint32_t)p.row_tiles - 1u) {
+                        hdr->done = 0;
+                        hdr->full_steps = hdr->full_steps + 1;
+                    }
+                }
+            } else {
+                record_timeout(p);
             }
-            tc_fence_before();
-            fence_proxy_async();
-            mbar_arrive(bar.a_full);
-            // count this unit; the last unit of a block to get here counts the full step
-            if (warp == 6 && lane == 0) {
-                const uint32_t prev = atomicAdd(&hdr->done, 1u);
-                if (prev == (uint32_t)p.row_tiles - 1u) {
-                    hdr->done = 0;
-                    hdr->full_steps = hdr->full_steps + 1;
+            // the staging of the next unit's previous Chat may overwrite the A region once the
+            // pass-2 MMAs of this unit have read it
+            if (issuer) {
+                const int un_next = u + gridDim.x;
+                bool ok = mbar_wait(p2_done, ui & 1u, abort_flag);
+                if (ok && un_next < p.units) {
+                    const Unit x = decode_unit(p, un_next);
+                    if (*(volatile uint32_t *)&header_of(p, x.b)->full_steps != 0) request_chat(x);
                 }
             }
+            __syncwarp();
         }
     }
 
@@ -642,9 +767,9 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// bf16 tensor (inner, rows, blocks) with byte pitches; box (box_inner, box_rows, 1)
+// bf16 (or fp32: elem = 4) tensor (inner, rows, blocks) with byte pitches; box (box_inner, box_rows, 1)
 int make_map(CUtensorMap *m, const void *base, uint64_t inner, uint64_t rows, uint64_t blocks, uint64_t row_pitch,
-             uint64_t block_pitch, uint32_t box_inner, uint32_t box_rows) {
+             uint64_t block_pitch, uint32_t box_inner, uint32_t box_rows, uint32_t elem = 2) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return SVDCACHE_ERR_CUDA;
     const cuuint64_t dims[3] = {inner, rows, blocks};
@@ -653,11 +778,11 @@ int make_map(CUtensorMap *m, const void *base, uint64_t inner, uint64_t rows, ui
     const cuuint64_t strides[2] = {row_pitch, block_pitch};
     const cuuint32_t box[3] = {box_inner, box_rows, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
-    const uint32_t inner_bytes = box_inner * 2;
+    const uint32_t inner_bytes = box_inner * elem;
     const CUtensorMapSwizzle sw = inner_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
                                   : inner_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
                                                       : CU_TENSOR_MAP_SWIZZLE_32B;
-    const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+    const CUresult r = fn(m, elem == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? SVDCACHE_OK : SVDCACHE_ERR_CUDA;
@@ -676,22 +801,15 @@ int num_sms() {
 
 constexpr size_t kSmemBudget = 227 * 1024;
 
-bool fill_params(const StepArgs &a, UmmaParams &p, int want_a_bufs) {
+bool fill_params(const StepArgs &a, UmmaParams &p) {
     p.N = a.N; p.D = a.D; p.k = a.k; p.nblocks = a.nblocks;
     p.row_tiles = (int)((a.N + kTileRows - 1) / kTileRows);
     p.chunks_total = (a.D + kTileCols - 1) / kTileCols;
-    p.kb_elems = a.k < 64 ? a.k : 64;
+    p.kb_elems = a.k < 64 ? a.k : 64;            // K block of the rank dimension: one swizzled row
     p.kb_bytes = p.kb_elems * 2;
     p.nkb = a.k / p.kb_elems;
     p.a_half_bytes = (uint32_t)kTileRows * a.k * 2;
     p.a_bytes = 2 * p.a_half_bytes;
-    p.v_bytes = (uint32_t)kTileCols * a.k * 2;
-    p.stage_bytes = kTileBytes + ((p.v_bytes + 1023u) & ~1023u);
-    const size_t avail = kSmemBudget - 1024 /*alignment*/ - kBarBytes - 64;
-    p.a_bufs = (want_a_bufs == 2 && 2 * (size_t)p.a_bytes + 4 * (size_t)p.stage_bytes <= avail) ? 2 : 1;
-    if ((size_t)p.a_bufs * p.a_bytes + 2 * (size_t)p.stage_bytes > avail) return false;
-    p.stages = (int)((avail - (size_t)p.a_bufs * p.a_bytes) / p.stage_bytes);
-    if (p.stages > kMaxStages) p.stages = kMaxStages;
     p.state = (char *)a.state;
     p.state_stride = a.state_stride;
     {
@@ -704,9 +822,7 @@ bool fill_params(const StepArgs &a, UmmaParams &p, int want_a_bufs) {
     return true;
 }
 
-// Cached step: shared memory = A tile(s) | basis-slice ring | R ring | barriers.
-bool fill_cached(const StepArgs &a, UmmaParams &p) {
-    if (!fill_params(a, p, 1)) return false;
+void fill_groups(const StepArgs &a, UmmaParams &p) {
     p.gc = 16384 / (kTileCols * a.k);            // basis slice (gc * 64 x k bf16) of at most 32 KB
     if (p.gc > 4) p.gc = 4;                      // MMA N = gc * 64 <= 256
     if (p.gc < 1) p.gc = 1;
@@ -714,6 +830,33 @@ bool fill_cached(const StepArgs &a, UmmaParams &p) {
     p.acc_stages = 512 / p.acc_cols < kAccStages ? 512 / p.acc_cols : kAccStages;
     p.vslice_bytes = (uint32_t)p.gc * kTileCols * a.k * 2;
     p.v_slots = kMaxVSlots;
+}
+
+// Full step: shared memory = A operand region (+ Chat staging when k < 64) | basis ring | F ring | barriers.
+bool fill_full(const StepArgs &a, UmmaParams &p) {
+    if (!fill_params(a, p)) return false;
+    fill_groups(a, p);
+    p.nacc = 256 / a.k < 4 ? 256 / a.k : 4;
+    if (p.nacc < 1) p.nacc = 1;
+    p.chat_stage_off = a.k >= 64 ? 0u : p.a_bytes;
+    p.a_region_bytes = p.a_bytes + (a.k >= 64 ? 0u : (uint32_t)kTileRows * a.k * 4u);
+    p.a_region_bytes = (p.a_region_bytes + 1023u) & ~1023u;
+    const size_t avail = kSmemBudget - 1024 /*alignment*/ - kBarBytes - 64;
+    const size_t fixed = (size_t)p.a_region_bytes + (size_t)p.v_slots * p.vslice_bytes;
+    if (fixed + 2 * (size_t)kTileBytes > avail) return false;
+    p.stages = (int)((avail - fixed) / kTileBytes);
+    if (p.stages > kMaxStages) p.stages = kMaxStages;
+    p.a_bufs = 1;
+    return true;
+}
+size_t smem_bytes_full(const UmmaParams &p) {
+    return 1024 + (size_t)p.a_region_bytes + (size_t)p.v_slots * p.vslice_bytes + (size_t)p.stages * kTileBytes +
+           kBarBytes + 64;
+}
+
+bool fill_cached(const StepArgs &a, UmmaParams &p) {
+    if (!fill_params(a, p)) return false;
+    fill_groups(a, p);
     const size_t avail = kSmemBudget - 1024 /*alignment*/ - kBarBytes - 64;
     const size_t fixed = (size_t)p.v_slots * p.vslice_bytes;
     p.a_bufs = (2 * (size_t)p.a_bytes + fixed + 6 * (size_t)kTileBytes <= avail) ? 2 : 1;
@@ -725,10 +868,6 @@ bool fill_cached(const StepArgs &a, UmmaParams &p) {
 size_t smem_bytes_cached(const UmmaParams &p) {
     return 1024 + (size_t)p.a_bufs * p.a_bytes + (size_t)p.v_slots * p.vslice_bytes + (size_t)p.stages * kTileBytes +
            kBarBytes + 64;
-}
-
-size_t smem_bytes(const UmmaParams &p) {
-    return 1024 + (size_t)p.a_bufs * p.a_bytes + (size_t)p.stages * p.stage_bytes + kBarBytes + 64;
 }
 
 bool shape_ok(const StepArgs &a) {
@@ -743,7 +882,7 @@ bool shape_ok(const StepArgs &a) {
 bool umma_supported(const StepArgs &a, bool full) {
     if (!shape_ok(a)) return false;
     UmmaParams p;
-    return full ? fill_params(a, p, 1) : fill_cached(a, p);
+    return full ? fill_full(a, p) : fill_cached(a, p);
 }
 
 int umma_cached_step(const StepArgs &a, cudaStream_t s) {
@@ -798,27 +937,30 @@ int umma_cached_step(const StepArgs &a, cudaStream_t s) {
 
 int umma_full_step(const StepArgs &a, cudaStream_t s) {
     UmmaParams p{};
-    if (!fill_params(a, p, 1)) return SVDCACHE_ERR_BAD_SHAPE;
+    if (!fill_full(a, p)) return SVDCACHE_ERR_BAD_SHAPE;
     p.dsplit = 1;
     p.chunks_per_slice = p.chunks_total;
     p.units = p.row_tiles * a.nblocks;
 
     const StateLayout SL = state_layout(a.N, a.D, a.k, a.dtype);
     const BasisLayout BL = basis_layout(a.D, a.k, a.dtype);
-    CUtensorMap tm_f, tm_vt, tm_v, tm_rout;
+    CUtensorMap tm_f, tm_vt, tm_v, tm_rout, tm_chat;
     int rc = make_map(&tm_f, a.F, a.D, a.N, a.nblocks, (uint64_t)a.ld * 2, a.F_stride, kTileCols, kTileRows);
     if (rc) return rc;
     rc = make_map(&tm_vt, (const char *)a.basis + BL.vt_bf16, a.D, a.k, a.nblocks, (uint64_t)a.D * 2,
                   a.basis_stride, kTileCols, a.k);
     if (rc) return rc;
     rc = make_map(&tm_v, (const char *)a.basis + BL.v_bf16, a.k, a.D, a.nblocks, (uint64_t)a.k * 2, a.basis_stride,
-                  p.kb_elems, kTileCols);
+                  p.kb_elems, p.gc * kTileCols);
     if (rc) return rc;
     rc = make_map(&tm_rout, (char *)a.state + SL.r, a.D, a.N, a.nblocks, (uint64_t)a.D * 2, a.state_stride,
-                  kTileCols, kTileRows);
+                  kTileCols, kSlabRows);
+    if (rc) return rc;
+    rc = make_map(&tm_chat, (char *)a.state + SL.chat, a.k, a.N, a.nblocks, (uint64_t)a.k * 4, a.state_stride,
+                  a.k < 32 ? a.k : 32, kTileRows, 4);
     if (rc) return rc;
 
-    const size_t smem = smem_bytes(p);
+    const size_t smem = smem_bytes_full(p);
     static bool attr_set = false;
     if (!attr_set) {
         rc = record_cuda(cudaFuncSetAttribute(umma_full_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -827,7 +969,7 @@ int umma_full_step(const StepArgs &a, cudaStream_t s) {
         attr_set = true;
     }
     const int grid = p.units < num_sms() ? p.units : num_sms();
-    umma_full_kernel<<<grid, kThreadsUmma, smem, s>>>(tm_f, tm_vt, tm_v, tm_rout, p);
+    umma_full_kernel<<<grid, kThreadsFull, smem, s>>>(tm_f, tm_vt, tm_v, tm_rout, tm_chat, p);
     count_launch();
     return check_last_launch();
 }
