@@ -18,6 +18,10 @@ namespace svdc {
 
 using namespace sm100;
 
+#ifdef SVDC_TRACE
+__device__ unsigned long long g_trace[148 * 16 * 8];
+#endif
+
 namespace {
 
 constexpr int kTileRows = 128;      // MMA M
@@ -37,7 +41,6 @@ struct UmmaParams {
     uint32_t a_half_bytes, a_bytes;
     int gc, acc_stages, acc_cols, v_slots;   // chunks per MMA group, TMEM ring, basis ring
     uint32_t vslice_bytes;
-    int nacc;                                // full step: pass-1 accumulators
     uint32_t a_region_bytes, chat_stage_off; // full step: A operand (+ Chat staging when k < 64)
     char *state;
     size_t state_stride, chat_off, ophi_off, oplo_off;
@@ -342,21 +345,22 @@ done:
 //
 // A unit is one 128-row tile of one block.
 //   Pass 1 streams the tile's F in 64-column chunks and accumulates C (128 x k, fp32) in
-//     TMEM: A = F chunk, B = matching columns of V_k^T.  Consecutive chunks go to different
-//     accumulators (up to four), so their dependent MMA chains overlap; the C warps add them.
+//     TMEM: A = F chunk, B = matching columns of V_k^T.
 //   The C warps read C from TMEM, apply the EMA against the previous Chat (staged by TMA in
 //     the A-operand region and converted in place), write Chat, and leave C as a split-bf16
 //     A operand in shared memory -- which also goes out, as it is, as the state's operand copy.
 //   Pass 2 streams the same F chunks again, last group first (the most recently read ones
 //     are the likeliest to sit in L2), with V_k slices of gc*64 rows: C V_k^T per group in
 //     TMEM, and the epilogue stores R = F - C V_k^T through TMA.
-// The pass-1 accumulators overlay the pass-2 accumulator ring, so pass 1 of a unit starts
-// once the epilogue has drained the previous unit.
+// TMEM holds C in columns [0, k) and the pass-2 accumulator ring after it, so pass 1 of the
+// next unit runs while the epilogue still drains this one.  The producer requests each basis
+// slice one group ahead of the F chunks that go with it.
 //
-// Warp roles (448 threads): 0 = TMA producer, 1 = MMA issuer (+ TMEM owner), 2..9 = two
-// epilogue groups of four warps, 10..13 = C warps.
+// Warp roles (320 threads): 0 = TMA producer, 1 = MMA issuer (+ TMEM owner), 2..5 = epilogue
+// group 0, 6..9 = C warps, which turn into epilogue group 1 once the A operand is written
+// (pass 2 cannot start before that, so the two jobs never overlap).
 // ======================================================================================
-constexpr int kThreadsFull = 448;
+constexpr int kThreadsFull = 320;
 constexpr uint32_t kBlk32Bytes = kTileRows * 128u;   // 16 KB: 128 rows x 32 fp32 (or x 64 bf16)
 
 // 32 consecutive coefficients of one row: EMA against `prev`, global stores, split-bf16 pack.
@@ -410,6 +414,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(gen_base + (bar.tmem_slot - base));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    SVDC_TRACE_DECL
     const uint32_t tmem_cols = 512;
     const int CT = p.chunks_total;
     const int G = (CT + p.gc - 1) / p.gc;               // groups per pass
@@ -445,35 +450,65 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
         // ------------------------------------------------------------ TMA producer ---
         if (lane == 0) {
             const uint64_t pol_keep = policy_evict_last(), pol_drop = policy_evict_first();
-            uint32_t it = 0, iv = 0;   // F chunks, basis slices requested so far
-            for (int u = blockIdx.x; u < p.units; u += gridDim.x) {
-                const Unit un = decode_unit(p, u);
-                for (int pass = 0; pass < 2; ++pass) {
-                    for (int g = 0; g < G; ++g, ++iv) {
-                        const int cg = (pass == 0 ? g : G - 1 - g) * p.gc;
-                        const int ce = min(cg + p.gc, CT);
-                        const uint32_t vs = iv % p.v_slots;
-                        if (!mbar_wait(bar.v_empty + 8 * vs, ((iv / p.v_slots) & 1u) ^ 1u, abort_flag)) { record_timeout(p); goto done; }
+            // Two request streams share this thread: F chunks (ring of p.stages slots) and basis
+            // slices (ring of p.v_slots slots), both in (unit, pass, group) order.  Neither may
+            // hold the other up -- a blocked F ring must not delay the next basis slice, and the
+            // other way round -- so the thread polls both rings without blocking.
+            struct Step { int u, pass, g; };
+            auto next_step = [&](Step x) {
+                if (++x.g == G) { x.g = 0; if (++x.pass == 2) { x.pass = 0; x.u += gridDim.x; } }
+                return x;
+            };
+            Step vcur{(int)blockIdx.x, 0, 0}, fcur{(int)blockIdx.x, 0, 0};
+            uint32_t iv = 0, it = 0;   // basis slices, F chunks requested so far
+            int fc = 0;                // next chunk of fcur's group (offset within the group)
+            long long t_idle = clock64();
+            SVDC_TRACE_MARK(tp);
+            while (fcur.u < p.units || vcur.u < p.units) {
+                bool progress = false;
+                if (vcur.u < p.units) {
+                    const uint32_t vs = iv % p.v_slots;
+                    if (mbar_test_wait(bar.v_empty + 8 * vs, ((iv / p.v_slots) & 1u) ^ 1u)) {
+                        const Unit un = decode_unit(p, vcur.u);
+                        const int cg = (vcur.pass == 0 ? vcur.g : G - 1 - vcur.g) * p.gc;
                         const uint32_t vdst = v_base0 + vs * p.vslice_bytes;
                         mbar_arrive_expect_tx(bar.v_full + 8 * vs, p.vslice_bytes);
-                        if (pass == 0) {   // V_k^T columns of each chunk: gc boxes of k rows x 64
+                        if (vcur.pass == 0) {   // V_k^T columns of each chunk: gc boxes of k rows x 64
                             for (int j = 0; j < p.gc; ++j)
                                 tma_load_3d(vdst + j * (p.k * 128), &tm_vt, bar.v_full + 8 * vs, (cg + j) * kTileCols, 0, un.b);
-                        } else {           // V_k rows of the group: one box of gc*64 rows per K block
+                        } else {                // V_k rows of the group: one box of gc*64 rows per K block
                             for (int kb = 0; kb < p.nkb; ++kb)
                                 tma_load_3d(vdst + kb * (p.gc * kTileCols * p.kb_bytes), &tm_v, bar.v_full + 8 * vs,
                                             kb * p.kb_elems, cg * kTileCols, un.b);
                         }
-                        for (int c = cg; c < ce; ++c, ++it) {
-                            const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                            if (!mbar_wait(bar.empty + 8 * s, ph ^ 1u, abort_flag)) { record_timeout(p); goto done; }
-                            mbar_arrive_expect_tx(bar.full + 8 * s, kTileBytes);
-                            tma_load_3d_hint(stage0 + s * kTileBytes, &tm_f, bar.full + 8 * s, c * kTileCols,
-                                             un.rt * kTileRows, un.b, pass == 0 ? pol_keep : pol_drop);
-                        }
+                        vcur = next_step(vcur);
+                        ++iv;
+                        progress = true;
                     }
                 }
+                if (fcur.u < p.units) {
+                    const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
+                    if (mbar_test_wait(bar.empty + 8 * s, ph ^ 1u)) {
+                        const Unit un = decode_unit(p, fcur.u);
+                        const int cg = (fcur.pass == 0 ? fcur.g : G - 1 - fcur.g) * p.gc;
+                        const int nsub = min(p.gc, CT - cg);
+                        mbar_arrive_expect_tx(bar.full + 8 * s, kTileBytes);
+                        tma_load_3d_hint(stage0 + s * kTileBytes, &tm_f, bar.full + 8 * s, (cg + fc) * kTileCols,
+                                         un.rt * kTileRows, un.b, fcur.pass == 0 ? pol_keep : pol_drop);
+                        ++it;
+                        if (++fc == nsub) { fc = 0; fcur = next_step(fcur); }
+                        progress = true;
+                    }
+                }
+                if (progress) {
+                    t_idle = clock64();
+                } else if (*abort_flag || clock64() - t_idle > kWaitCycles) {
+                    *abort_flag = 1;
+                    record_timeout(p);
+                    goto done;
+                }
             }
+            SVDC_TRACE_ADD(0, tp);
         }
     } else if (warp == 1) {
         // -------------------------------------------------------------- MMA issuer ---
@@ -483,43 +518,50 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
             const int ksteps = p.kb_elems / 16;
             const uint64_t a_desc0 = smem_desc_kmajor(a_base, p.kb_bytes);
             for (int u = blockIdx.x; u < p.units; u += gridDim.x, ++ui) {
-                // the pass-1 accumulators overlay the pass-2 ring: wait until it has drained
-                for (int as = 0; as < p.acc_stages; ++as) {
-                    const uint32_t uses = (ig + p.acc_stages - 1 - as) / p.acc_stages;   // uses of stage `as` so far
-                    if (!mbar_wait(bar.acc_empty + 8 * as, (uses & 1u) ^ 1u, abort_flag)) { record_timeout(p); goto done; }
-                }
-                tc_fence_after();
+                // C of the previous unit has been read out of TMEM: a_full(ui - 1) was awaited below
                 for (int g = 0; g < G; ++g, ++iv) {                 // pass 1: C_a += F_chunk (V^T chunk)^T
                     const int cg = g * p.gc, ce = min(cg + p.gc, CT);
                     const uint32_t vs = iv % p.v_slots;
+                    SVDC_TRACE_MARK(t0);
                     if (!mbar_wait(bar.v_full + 8 * vs, (iv / p.v_slots) & 1u, abort_flag)) { record_timeout(p); goto done; }
+                    SVDC_TRACE_ADD(0, t0);
                     for (int c = cg; c < ce; ++c, ++it) {
                         const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
+                        SVDC_TRACE_MARK(t1);
                         if (!mbar_wait(bar.full + 8 * s, ph, abort_flag)) { record_timeout(p); goto done; }
+                        SVDC_TRACE_ADD(1, t1);
                         tc_fence_after();
+                        SVDC_TRACE_MARK(t2);
                         const uint64_t fd = smem_desc_kmajor(stage0 + s * kTileBytes, 128);
                         const uint64_t vd = smem_desc_kmajor(v_base0 + vs * p.vslice_bytes + (c - cg) * (p.k * 128), 128);
-                        const uint32_t d = tmem_base + (uint32_t)(c % p.nacc) * p.k;
 #pragma unroll
                         for (int ks = 0; ks < kTileCols / 16; ++ks)
-                            mma_bf16_ss(d, fd + 2 * ks, vd + 2 * ks, idesc1, (c >= p.nacc || ks > 0) ? 1u : 0u);
+                            mma_bf16_ss(tmem_base, fd + 2 * ks, vd + 2 * ks, idesc1, (c | ks) != 0 ? 1u : 0u);
                         mma_commit(bar.empty + 8 * s);
                         mbar_arrive_n(bar.empty + 8 * s, 3);   // pass 1 has no slab stores: their three other arrivals
+                        SVDC_TRACE_ADD(2, t2);
                     }
                     mma_commit(bar.v_empty + 8 * vs);
                 }
                 mma_commit(bar.c_full);
+                SVDC_TRACE_MARK(t3);
                 if (!mbar_wait(bar.a_full, ui & 1u, abort_flag)) { record_timeout(p); goto done; }
+                SVDC_TRACE_ADD(3, t3);
                 tc_fence_after();
                 for (int g = 0; g < G; ++g, ++iv, ++ig) {           // pass 2: acc = C (V slice)^T
                     const int cg = (G - 1 - g) * p.gc;
                     const int nsub = min(p.gc, CT - cg);
                     const uint32_t vs = iv % p.v_slots, as = ig % p.acc_stages;
+                    SVDC_TRACE_MARK(t4);
                     if (!mbar_wait(bar.v_full + 8 * vs, (iv / p.v_slots) & 1u, abort_flag)) { record_timeout(p); goto done; }
+                    SVDC_TRACE_ADD(4, t4);
+                    SVDC_TRACE_MARK(t5);
                     if (!mbar_wait(bar.acc_empty + 8 * as, ((ig / p.acc_stages) & 1u) ^ 1u, abort_flag)) { record_timeout(p); goto done; }
+                    SVDC_TRACE_ADD(5, t5);
                     tc_fence_after();
+                    SVDC_TRACE_MARK(t6);
                     const uint32_t idesc = idesc_bf16(kTileRows, nsub * kTileCols);
-                    const uint32_t d_tmem = tmem_base + as * p.acc_cols;
+                    const uint32_t d_tmem = tmem_base + p.k + as * p.acc_cols;
                     const uint64_t v_desc0 = smem_desc_kmajor(v_base0 + vs * p.vslice_bytes, p.kb_bytes);
                     uint32_t acc = 0;
                     for (int part = 0; part < 2; ++part)
@@ -533,74 +575,24 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                         }
                     mma_commit(bar.v_empty + 8 * vs);
                     mma_commit(bar.acc_full + 8 * as);
+                    SVDC_TRACE_ADD(6, t6);
                 }
                 mma_commit(p2_done);
                 it += CT;   // pass-2 slots are consumed by the epilogue alone
             }
         }
-    } else if (warp < 10) {
-        // ------------------------------------------- epilogue: R = F - C V_k^T, TMA store ---
+    } else {
+        // --------------- epilogue (R = F - C V_k^T, TMA store) and, for warps 6..9, the C job ---
         const int q = warp & 3, row = q * kSlabRows + lane;
         const uint32_t grp = (uint32_t)(warp - 2) >> 2;
-        uint32_t it = 0, ig = 0;
-        for (int u = blockIdx.x; u < p.units; u += gridDim.x) {
-            const Unit un = decode_unit(p, u);
-            const int slab_row0 = un.rt * kTileRows + q * kSlabRows;
-            const bool slab_live = (int64_t)slab_row0 < p.N;
-            it += CT;   // pass-1 slots are consumed by the MMA warp alone
-            for (int g = 0; g < G; ++g, ++ig) {
-                const int cg = (G - 1 - g) * p.gc;
-                const int nsub = min(p.gc, CT - cg);
-                const uint32_t as = ig % p.acc_stages, aph = (ig / p.acc_stages) & 1u;
-                for (int j = 0; j < nsub; ++j, ++it) {
-                    if ((it & 1u) != grp) continue;
-                    const int c = cg + j;
-                    const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                    bool ok = mbar_wait(bar.acc_full + 8 * as, aph, abort_flag);
-                    ok = ok && mbar_wait(bar.full + 8 * s, ph, abort_flag);
-                    if (!__all_sync(0xFFFFFFFFu, ok)) { record_timeout(p); goto done; }
-                    tc_fence_after();
-                    const uint32_t tile = stage0 + s * kTileBytes + (uint32_t)row * 128u;
-                    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + as * p.acc_cols + j * kTileCols;
-                    uint32_t acc0[32], acc1[32];
-                    tmem_ld_32x32(taddr, acc0);
-                    tmem_ld_32x32(taddr + 32, acc1);
-                    uint4 t[8];
-#pragma unroll
-                    for (int cc = 0; cc < 8; ++cc) t[cc] = lds128(tile + (((uint32_t)cc) ^ ((uint32_t)row & 7u)) * 16u);
-                    tmem_wait_ld();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_n(bar.acc_empty + 8 * as, j == nsub - 1 ? 1u + (uint32_t)(p.gc - nsub) : 1u);
-#pragma unroll
-                    for (int cc = 0; cc < 8; ++cc)
-                        sts128(tile + (((uint32_t)cc) ^ ((uint32_t)row & 7u)) * 16u,
-                               combine_chunk<true>(t[cc], cc < 4 ? acc0 + cc * 8 : acc1 + (cc - 4) * 8));
-                    fence_proxy_async();
-                    __syncwarp();
-                    if (lane == 0) {
-                        if (slab_live)
-                            tma_store_3d(&tm_rout, stage0 + s * kTileBytes + (uint32_t)q * kSlabBytes, c * kTileCols,
-                                         slab_row0, un.b);
-                        tma_store_commit();
-                        tma_store_wait_read<0>();
-                        mbar_arrive(bar.empty + 8 * s);
-                    }
-                    __syncwarp();
-                }
-            }
-        }
-        if (lane == 0) tma_store_wait<0>();
-    } else {
-        // ------------- C warps: TMEM -> EMA -> Chat, split-bf16 A operand (+ its copy in the state) ---
-        const int q = warp & 3, row = q * 32 + lane;
+        const bool c_warp = grp == 1;
+        const bool issuer = (warp == 6 && lane == 0);
         const float beta = p.beta, omb = 1.0f - p.beta;
-        const bool issuer = (warp == 10 && lane == 0);
         const uint32_t chat_row_bytes = p.k >= 32 ? 128u : (uint32_t)p.k * 4u;
         const int nblk = (p.k + 31) / 32;
-        const int nacc_used = CT < p.nacc ? CT : p.nacc;
-        uint32_t ui = 0, nchat = 0;   // units done; Chat tiles consumed
-        bool alive = true;
+        uint32_t it = 0, ig = 0, ui = 0, nchat = 0;   // F chunks, pass-2 groups, units, Chat tiles consumed
+        int prev_slot = -1;                           // slot whose slab store may still be reading
+        const bool defer_release = p.stages >= 4;
 
         auto request_chat = [&](const Unit &x) {   // previous Chat of unit x -> staging, by TMA
             mbar_arrive_expect_tx(chat_full, (uint32_t)kTileRows * p.k * 4u);
@@ -613,15 +605,20 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
         }
         for (int u = blockIdx.x; u < p.units; u += gridDim.x, ++ui) {
             const Unit un = decode_unit(p, u);
-            StateHeader *hdr = header_of(p, un.b);
-            const bool first = *(volatile uint32_t *)&hdr->full_steps == 0;
-            if (alive && !first) {
-                alive = __all_sync(0xFFFFFFFFu, mbar_wait(chat_full, nchat & 1u, abort_flag));
-                ++nchat;
-            }
-            if (alive) alive = __all_sync(0xFFFFFFFFu, mbar_wait(bar.c_full, ui & 1u, abort_flag));
-            if (alive) {
+            if (c_warp) {
+                // ---- C job: TMEM -> EMA -> Chat, split-bf16 A operand (+ the state's operand copy)
+                StateHeader *hdr = header_of(p, un.b);
+                const bool first = *(volatile uint32_t *)&hdr->full_steps == 0;
+                bool ok = true;
+                SVDC_TRACE_MARK(c0);
+                if (!first) { ok = mbar_wait(chat_full, nchat & 1u, abort_flag); ++nchat; }
+                SVDC_TRACE_ADD(0, c0);
+                SVDC_TRACE_MARK(c1);
+                ok = ok && mbar_wait(bar.c_full, ui & 1u, abort_flag);
+                if (!__all_sync(0xFFFFFFFFu, ok)) { record_timeout(p); goto done; }
+                SVDC_TRACE_ADD(1, c1);
                 tc_fence_after();
+                SVDC_TRACE_MARK(c2);
                 const int64_t n = (int64_t)un.rt * kTileRows + row;
                 const bool row_live = n < p.N;
                 char *st_b = p.state + (size_t)un.b * p.state_stride;
@@ -651,12 +648,6 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                             tmem_wait_ld();
 #pragma unroll
                             for (int i = 0; i < 32; ++i) cs[i] = __uint_as_float(tmp[i]);
-                            for (int a = 1; a < nacc_used; ++a) {
-                                tmem_ld_32x32(taddr + a * p.k + col0, tmp);
-                                tmem_wait_ld();
-#pragma unroll
-                                for (int i = 0; i < 32; ++i) cs[i] += __uint_as_float(tmp[i]);
-                            }
                         }
                         float ch[32];
                         if (first) {
@@ -671,18 +662,6 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
 #pragma unroll
                             for (int i = 0; i < 32; ++i) ch[i] = fmaf(beta, ch[i], omb * cs[i]);
                         }
-                        if (row_live) {
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) {
-                                if (i * 4 < ncols) {
-                                    *reinterpret_cast<float4 *>(chat_g + col0 + 4 * i) =
-                                        make_float4(ch[4 * i], ch[4 * i + 1], ch[4 * i + 2], ch[4 * i + 3]);
-                                    if (cout_g)
-                                        *reinterpret_cast<float4 *>(cout_g + col0 + 4 * i) =
-                                            make_float4(cs[4 * i], cs[4 * i + 1], cs[4 * i + 2], cs[4 * i + 3]);
-                                }
-                            }
-                        }
                         // split-bf16 operand of C (not of Chat) for pass 2 ...
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
@@ -694,8 +673,18 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                                 sts128(lo_row + chunk, lo);
                             }
                         }
-                        // ... while the state keeps the split of the new Chat
                         if (row_live) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                if (i * 4 < ncols) {
+                                    *reinterpret_cast<float4 *>(chat_g + col0 + 4 * i) =
+                                        make_float4(ch[4 * i], ch[4 * i + 1], ch[4 * i + 2], ch[4 * i + 3]);
+                                    if (cout_g)
+                                        *reinterpret_cast<float4 *>(cout_g + col0 + 4 * i) =
+                                            make_float4(cs[4 * i], cs[4 * i + 1], cs[4 * i + 2], cs[4 * i + 3]);
+                                }
+                            }
+                            // ... while the state keeps the split of the new Chat
                             __nv_bfloat16 *ohi = reinterpret_cast<__nv_bfloat16 *>(st_b + p.ophi_off) + n * p.k + col0;
                             __nv_bfloat16 *olo = reinterpret_cast<__nv_bfloat16 *>(st_b + p.oplo_off) + n * p.k + col0;
 #pragma unroll
@@ -713,6 +702,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                 tc_fence_before();
                 fence_proxy_async();
                 mbar_arrive(bar.a_full);
+                SVDC_TRACE_ADD(2, c2);
                 // count this unit; the last unit of a block to get here counts the full step
                 if (issuer) {
                     const uint32_t prev = atomicAdd(&hdr->done, 1u);
@@ -721,14 +711,79 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                         hdr->full_steps = hdr->full_steps + 1;
                     }
                 }
-            } else {
-                record_timeout(p);
             }
-            // the staging of the next unit's previous Chat may overwrite the A region once the
-            // pass-2 MMAs of this unit have read it
+            // ---- epilogue duty for this group's chunks of pass 2
+            const int slab_row0 = un.rt * kTileRows + q * kSlabRows;
+            const bool slab_live = (int64_t)slab_row0 < p.N;
+            it += CT;   // pass-1 slots are consumed by the MMA warp alone
+            for (int g = 0; g < G; ++g, ++ig) {
+                const int cg = (G - 1 - g) * p.gc;
+                const int nsub = min(p.gc, CT - cg);
+                const uint32_t as = ig % p.acc_stages, aph = (ig / p.acc_stages) & 1u;
+                for (int j = 0; j < nsub; ++j, ++it) {
+                    if ((it & 1u) != grp) continue;
+                    const int c = cg + j;
+                    const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
+                    SVDC_TRACE_MARK(e3);
+                    bool ok = mbar_wait(bar.acc_full + 8 * as, aph, abort_flag);
+                    SVDC_TRACE_ADD(3, e3);
+                    SVDC_TRACE_MARK(e4);
+                    ok = ok && mbar_wait(bar.full + 8 * s, ph, abort_flag);
+                    if (!__all_sync(0xFFFFFFFFu, ok)) { record_timeout(p); goto done; }
+                    SVDC_TRACE_ADD(4, e4);
+                    tc_fence_after();
+                    SVDC_TRACE_MARK(e5);
+                    const uint32_t tile = stage0 + s * kTileBytes + (uint32_t)row * 128u;
+                    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + p.k + as * p.acc_cols + j * kTileCols;
+                    uint32_t acc0[32], acc1[32];
+                    tmem_ld_32x32(taddr, acc0);
+                    tmem_ld_32x32(taddr + 32, acc1);
+                    uint4 t[8];
+#pragma unroll
+                    for (int cc = 0; cc < 8; ++cc) t[cc] = lds128(tile + (((uint32_t)cc) ^ ((uint32_t)row & 7u)) * 16u);
+                    tmem_wait_ld();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_n(bar.acc_empty + 8 * as, j == nsub - 1 ? 1u + (uint32_t)(p.gc - nsub) : 1u);
+#pragma unroll
+                    for (int cc = 0; cc < 8; ++cc)
+                        sts128(tile + (((uint32_t)cc) ^ ((uint32_t)row & 7u)) * 16u,
+                               combine_chunk<true>(t[cc], cc < 4 ? acc0 + cc * 8 : acc1 + (cc - 4) * 8));
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (slab_live)
+                            tma_store_3d(&tm_rout, stage0 + s * kTileBytes + (uint32_t)q * kSlabBytes, c * kTileCols,
+                                         slab_row0, un.b);
+                        tma_store_commit();
+                        // the slot goes back once its store has read it: checked one chunk late, so
+                        // the warp does not sit out the store it has just issued
+                        if (!defer_release) {   // a ring this short cannot lend a slot per warp
+                            tma_store_wait_read<0>();
+                            mbar_arrive(bar.empty + 8 * s);
+                        } else {
+                            if (prev_slot >= 0) {
+                                tma_store_wait_read<1>();
+                                mbar_arrive(bar.empty + 8 * prev_slot);
+                            }
+                            prev_slot = (int)s;
+                        }
+                    }
+                    __syncwarp();
+                    SVDC_TRACE_ADD(5, e5);
+                    SVDC_TRACE_COUNT(6);
+                }
+            }
+            if (lane == 0 && prev_slot >= 0) {   // last chunk of the unit: release at once
+                tma_store_wait_read<0>();
+                mbar_arrive(bar.empty + 8 * prev_slot);
+                prev_slot = -1;
+            }
+            // Every accumulator of this unit has been read, so its pass-2 MMAs are complete and
+            // the A region is free: stage the next unit's previous Chat there.
             if (issuer) {
                 const int un_next = u + gridDim.x;
-                bool ok = mbar_wait(p2_done, ui & 1u, abort_flag);
+                const bool ok = mbar_wait(p2_done, ui & 1u, abort_flag);
                 if (ok && un_next < p.units) {
                     const Unit x = decode_unit(p, un_next);
                     if (*(volatile uint32_t *)&header_of(p, x.b)->full_steps != 0) request_chat(x);
@@ -736,9 +791,11 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
             }
             __syncwarp();
         }
+        if (lane == 0) tma_store_wait<0>();
     }
 
 done:
+    SVDC_TRACE_FLUSH(g_trace);
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -836,8 +893,11 @@ void fill_groups(const StepArgs &a, UmmaParams &p) {
 bool fill_full(const StepArgs &a, UmmaParams &p) {
     if (!fill_params(a, p)) return false;
     fill_groups(a, p);
-    p.nacc = 256 / a.k < 4 ? 256 / a.k : 4;
-    if (p.nacc < 1) p.nacc = 1;
+    // TMEM: C in columns [0, k), then the pass-2 ring; at least two ring stages
+    while (p.gc > 1 && a.k + 2 * p.gc * kTileCols > 512) --p.gc;
+    p.acc_cols = p.gc * kTileCols;
+    p.acc_stages = (512 - a.k) / p.acc_cols < kAccStages ? (512 - a.k) / p.acc_cols : kAccStages;
+    p.vslice_bytes = (uint32_t)p.gc * kTileCols * a.k * 2;
     p.chat_stage_off = a.k >= 64 ? 0u : p.a_bytes;
     p.a_region_bytes = p.a_bytes + (a.k >= 64 ? 0u : (uint32_t)kTileRows * a.k * 4u);
     p.a_region_bytes = (p.a_region_bytes + 1023u) & ~1023u;
@@ -878,6 +938,14 @@ bool shape_ok(const StepArgs &a) {
 }
 
 }  // namespace
+
+#ifdef SVDC_TRACE
+}  // namespace svdc
+extern "C" __attribute__((visibility("default"))) int svdcache_trace_dump(unsigned long long *host) {
+    return (int)cudaMemcpyFromSymbol(host, svdc::g_trace, sizeof(svdc::g_trace));
+}
+namespace svdc {
+#endif
 
 bool umma_supported(const StepArgs &a, bool full) {
     if (!shape_ok(a)) return false;

@@ -8,6 +8,28 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+// Optional cycle accounting for the warp-specialised kernels (compile with -DSVDC_TRACE):
+// each warp adds the cycles it spends in marked waits and sections to eight slots, and
+// lane 0 writes them to a device array at the end.  Compiled out otherwise.
+#ifdef SVDC_TRACE
+#define SVDC_TRACE_DECL unsigned long long trace_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}; const long long trace_t0 = clock64();
+#define SVDC_TRACE_MARK(v) const long long v = clock64()
+#define SVDC_TRACE_ADD(slot, v) trace_acc[slot] += (unsigned long long)(clock64() - (v))
+#define SVDC_TRACE_COUNT(slot) trace_acc[slot] += 1
+#define SVDC_TRACE_FLUSH(buf)                                                                     \
+    do {                                                                                          \
+        trace_acc[7] = (unsigned long long)(clock64() - trace_t0);                                \
+        if ((threadIdx.x & 31) == 0 && blockIdx.x < 148 && (threadIdx.x >> 5) < 16)               \
+            for (int i_ = 0; i_ < 8; ++i_) (buf)[(blockIdx.x * 16 + (threadIdx.x >> 5)) * 8 + i_] = trace_acc[i_]; \
+    } while (0)
+#else
+#define SVDC_TRACE_DECL
+#define SVDC_TRACE_MARK(v)
+#define SVDC_TRACE_ADD(slot, v)
+#define SVDC_TRACE_COUNT(slot)
+#define SVDC_TRACE_FLUSH(buf)
+#endif
+
 namespace svdc {
 namespace sm100 {
 
@@ -37,6 +59,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         "{\n\t"
         ".reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// non-blocking probe of a phase (try_wait may suspend the thread for a while; this does not)
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t"
         "}"
         : "=r"(ok)
