@@ -28,7 +28,7 @@ struct StateHeader {   // first 256 bytes of a state buffer
     uint32_t full_steps;   // full steps seen since the last reset
     int32_t status;        // sticky device status word (SVDCACHE_OK or an error code)
     uint32_t done;         // CTAs of the running full step that have finished
-    uint32_t pad;
+    uint32_t pad;          // which wait ran out first: site << 16 | CTA (diagnosis)
 };
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

@@ -95,8 +95,20 @@ __device__ __forceinline__ Unit decode_unit(const UmmaParams &p, int u) {
     return x;
 }
 
-__device__ __forceinline__ void record_timeout(const UmmaParams &p) {
-    atomicExch(&header_of(p, 0)->status, SVDCACHE_ERR_TIMEOUT);
+// A wait ran out: make the status sticky and leave a diagnosis in block 0's state header --
+// `pad` = (site of the first wait of the first CTA to give up) << 16 | that CTA, and, for
+// each warp of that CTA that got here, four words at byte 64 + 16 * warp: its own view of
+// the site and three progress counters of its role.
+__device__ __forceinline__ void record_timeout(const UmmaParams &p, volatile int *abort_flag, uint32_t c0 = 0,
+                                               uint32_t c1 = 0, uint32_t c2 = 0) {
+    StateHeader *h = header_of(p, 0);
+    atomicExch(&h->status, SVDCACHE_ERR_TIMEOUT);
+    const uint32_t mine = ((uint32_t)*abort_flag << 16) | (blockIdx.x & 0xFFFFu);
+    atomicCAS(&h->pad, 0u, mine);
+    if ((*(volatile uint32_t *)&h->pad & 0xFFFFu) == (blockIdx.x & 0xFFFFu) && (threadIdx.x & 31u) == 0u) {
+        uint32_t *w = reinterpret_cast<uint32_t *>(h) + 16 + 4 * (threadIdx.x >> 5);
+        w[0] = mine; w[1] = c0; w[2] = c1; w[3] = c2;
+    }
 }
 
 // 8 bf16 (one 16-byte chunk) combined with 8 fp32 accumulator values: out = sign*acc + tile
@@ -127,6 +139,20 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
 }
 __device__ __forceinline__ void sts64(uint32_t addr, uint32_t x, uint32_t y) {
     asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(addr), "r"(x), "r"(y) : "memory");
+}
+
+// Every epilogue warp waits for every accumulator of the ring, in order, and arrives on its
+// "empty" barrier once per group -- after reading its last chunk of the group, or at once if
+// the group holds none of its chunks.  A waiter that skipped a phase of an mbarrier could
+// take the completion of the phase before it for the one it wants (parities alias), and one
+// that does not gate the reuse could fall two phases behind; waiting on every phase and
+// gating each reuse rules both out.  Returns the index (within the group) of the last chunk
+// that belongs to epilogue group `grp`, or -1: chunk j of the group has running index
+// it0 + j and belongs to group (it0 + j) & 1.
+__device__ __forceinline__ int last_own_chunk(uint32_t it0, int nsub, uint32_t grp) {
+    int last = nsub - 1;
+    if (((it0 + (uint32_t)last) & 1u) != grp) --last;
+    return last;   // -1 when nsub == 1 and the only chunk is the other group's
 }
 
 // ======================================================================================
@@ -167,10 +193,10 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
     const uint32_t tmem_cols = 512;
 
     if (threadIdx.x == 0) {
-        // R slot: free again once the four slab stores have read it.  Accumulator: four
-        // arrivals (one per lane quarter) for each of the gc chunks of a group.
+        // R slot: free again once the four slab stores have read it.  Accumulator: one arrival
+        // from each of the eight epilogue warps per group (see group_share below).
         for (int s = 0; s < p.stages; ++s) { mbar_init(bar.full + 8 * s, 1); mbar_init(bar.empty + 8 * s, 4); }
-        for (int s = 0; s < p.acc_stages; ++s) { mbar_init(bar.acc_full + 8 * s, 1); mbar_init(bar.acc_empty + 8 * s, 4 * p.gc); }
+        for (int s = 0; s < p.acc_stages; ++s) { mbar_init(bar.acc_full + 8 * s, 1); mbar_init(bar.acc_empty + 8 * s, 8); }
         for (int s = 0; s < p.a_bufs; ++s) { mbar_init(bar.a_full + 8 * s, 1); mbar_init(bar.a_empty + 8 * s, 1); }
         for (int s = 0; s < p.v_slots; ++s) { mbar_init(bar.v_full + 8 * s, 1); mbar_init(bar.v_empty + 8 * s, 1); }
         *abort_flag = 0;
@@ -207,7 +233,7 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
                     u_a += gridDim.x;
                     if (*(volatile uint32_t *)&header_of(p, ux.b)->full_steps == 0) continue;
                     const uint32_t ab = ua % p.a_bufs;
-                    if (!mbar_wait(bar.a_empty + 8 * ab, ((ua / p.a_bufs) & 1u) ^ 1u, abort_flag)) { record_timeout(p); goto done; }
+                    if (!mbar_wait(bar.a_empty + 8 * ab, ((ua / p.a_bufs) & 1u) ^ 1u, abort_flag, 1)) { record_timeout(p, abort_flag); goto done; }
                     const uint32_t dst = a_base0 + ab * p.a_bytes;
                     mbar_arrive_expect_tx(bar.a_full + 8 * ab, p.a_bytes);
                     for (int kb = 0; kb < p.nkb; ++kb) {
@@ -221,7 +247,7 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
                 ++ui;
                 for (int cg = un.c0; cg < un.c1; cg += p.gc, ++ig) {
                     const uint32_t vs = ig % p.v_slots;
-                    if (!mbar_wait(bar.v_empty + 8 * vs, ((ig / p.v_slots) & 1u) ^ 1u, abort_flag)) { record_timeout(p); goto done; }
+                    if (!mbar_wait(bar.v_empty + 8 * vs, ((ig / p.v_slots) & 1u) ^ 1u, abort_flag, 2)) { record_timeout(p, abort_flag); goto done; }
                     const uint32_t vdst = v_base0 + vs * p.vslice_bytes;
                     mbar_arrive_expect_tx(bar.v_full + 8 * vs, p.vslice_bytes);
                     for (int kb = 0; kb < p.nkb; ++kb)
@@ -230,7 +256,7 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
                     const int ce = min(cg + p.gc, un.c1);
                     for (int c = cg; c < ce; ++c, ++it) {
                         const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                        if (!mbar_wait(bar.empty + 8 * s, ph ^ 1u, abort_flag)) { record_timeout(p); goto done; }
+                        if (!mbar_wait(bar.empty + 8 * s, ph ^ 1u, abort_flag, 3)) { record_timeout(p, abort_flag); goto done; }
                         mbar_arrive_expect_tx(bar.full + 8 * s, kTileBytes);
                         tma_load_3d(stage0 + s * kTileBytes, &tm_r, bar.full + 8 * s, c * kTileCols, un.rt * kTileRows, un.b);
                     }
@@ -246,13 +272,13 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
                 const Unit un = decode_unit(p, u);
                 if (*(volatile uint32_t *)&header_of(p, un.b)->full_steps == 0) continue;
                 const uint32_t ab = ui % p.a_bufs;
-                if (!mbar_wait(bar.a_full + 8 * ab, (ui / p.a_bufs) & 1u, abort_flag)) { record_timeout(p); goto done; }
+                if (!mbar_wait(bar.a_full + 8 * ab, (ui / p.a_bufs) & 1u, abort_flag, 4)) { record_timeout(p, abort_flag); goto done; }
                 const uint64_t a_desc0 = smem_desc_kmajor(a_base0 + ab * p.a_bytes, p.kb_bytes);
                 for (int cg = un.c0; cg < un.c1; cg += p.gc, ++ig) {
                     const uint32_t vs = ig % p.v_slots, as = ig % p.acc_stages;
                     const int nsub = min(p.gc, un.c1 - cg);
-                    if (!mbar_wait(bar.v_full + 8 * vs, (ig / p.v_slots) & 1u, abort_flag)) { record_timeout(p); goto done; }
-                    if (!mbar_wait(bar.acc_empty + 8 * as, ((ig / p.acc_stages) & 1u) ^ 1u, abort_flag)) { record_timeout(p); goto done; }
+                    if (!mbar_wait(bar.v_full + 8 * vs, (ig / p.v_slots) & 1u, abort_flag, 5)) { record_timeout(p, abort_flag); goto done; }
+                    if (!mbar_wait(bar.acc_empty + 8 * as, ((ig / p.acc_stages) & 1u) ^ 1u, abort_flag, 6)) { record_timeout(p, abort_flag); goto done; }
                     tc_fence_after();
                     const uint32_t idesc = idesc_bf16(kTileRows, nsub * kTileCols);
                     const uint32_t d_tmem = tmem_base + as * p.acc_cols;
@@ -288,13 +314,14 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
             for (int cg = un.c0; cg < un.c1; cg += p.gc, ++ig) {
                 const uint32_t as = ig % p.acc_stages, aph = (ig / p.acc_stages) & 1u;
                 const int nsub = min(p.gc, un.c1 - cg);
+                const int last_own = last_own_chunk(it, nsub, grp);
+                if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar.acc_full + 8 * as, aph, abort_flag, 7))) { record_timeout(p, abort_flag); goto done; }
+                if (last_own < 0 && lane == 0) mbar_arrive(bar.acc_empty + 8 * as);
                 for (int j = 0; j < nsub; ++j, ++it) {
                     if ((it & 1u) != grp) continue;
                     const int c = cg + j;
                     const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                    bool ok = mbar_wait(bar.acc_full + 8 * as, aph, abort_flag);
-                    ok = ok && mbar_wait(bar.full + 8 * s, ph, abort_flag);
-                    if (!__all_sync(0xFFFFFFFFu, ok)) { record_timeout(p); goto done; }
+                    if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar.full + 8 * s, ph, abort_flag, 8))) { record_timeout(p, abort_flag); goto done; }
                     tc_fence_after();
                     const uint32_t tile = stage0 + s * kTileBytes + (uint32_t)row * 128u;
                     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + as * p.acc_cols + j * kTileCols;
@@ -307,9 +334,7 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
                     tmem_wait_ld();
                     tc_fence_before();
                     __syncwarp();
-                    // this quarter's share of the group's accumulator is in registers; the last
-                    // chunk of a short group also arrives for the chunks the group does not have
-                    if (lane == 0) mbar_arrive_n(bar.acc_empty + 8 * as, j == nsub - 1 ? 1u + (uint32_t)(p.gc - nsub) : 1u);
+                    if (lane == 0 && j == last_own) mbar_arrive(bar.acc_empty + 8 * as);   // this warp is done with the group
 #pragma unroll
                     for (int cc = 0; cc < 8; ++cc)
                         sts128(tile + (((uint32_t)cc) ^ ((uint32_t)row & 7u)) * 16u,
@@ -423,7 +448,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) { mbar_init(bar.full + 8 * s, 1); mbar_init(bar.empty + 8 * s, 4); }
-        for (int s = 0; s < p.acc_stages; ++s) { mbar_init(bar.acc_full + 8 * s, 1); mbar_init(bar.acc_empty + 8 * s, 4 * p.gc); }
+        for (int s = 0; s < p.acc_stages; ++s) { mbar_init(bar.acc_full + 8 * s, 1); mbar_init(bar.acc_empty + 8 * s, 8); }
         for (int s = 0; s < p.v_slots; ++s) { mbar_init(bar.v_full + 8 * s, 1); mbar_init(bar.v_empty + 8 * s, 1); }
         mbar_init(bar.a_full, 128);
         mbar_init(chat_full, 1);
@@ -503,8 +528,8 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                 if (progress) {
                     t_idle = clock64();
                 } else if (*abort_flag || clock64() - t_idle > kWaitCycles) {
-                    *abort_flag = 1;
-                    record_timeout(p);
+                    atomicCAS(const_cast<int *>(abort_flag), 0, 100);
+                    record_timeout(p, abort_flag, it, iv, (uint32_t)(fcur.pass * 100 + fcur.g) << 16 | (uint32_t)(vcur.pass * 100 + vcur.g));
                     goto done;
                 }
             }
@@ -523,12 +548,12 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                     const int cg = g * p.gc, ce = min(cg + p.gc, CT);
                     const uint32_t vs = iv % p.v_slots;
                     SVDC_TRACE_MARK(t0);
-                    if (!mbar_wait(bar.v_full + 8 * vs, (iv / p.v_slots) & 1u, abort_flag)) { record_timeout(p); goto done; }
+                    if (!mbar_wait(bar.v_full + 8 * vs, (iv / p.v_slots) & 1u, abort_flag, 9)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
                     SVDC_TRACE_ADD(0, t0);
                     for (int c = cg; c < ce; ++c, ++it) {
                         const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
                         SVDC_TRACE_MARK(t1);
-                        if (!mbar_wait(bar.full + 8 * s, ph, abort_flag)) { record_timeout(p); goto done; }
+                        if (!mbar_wait(bar.full + 8 * s, ph, abort_flag, 10)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
                         SVDC_TRACE_ADD(1, t1);
                         tc_fence_after();
                         SVDC_TRACE_MARK(t2);
@@ -545,7 +570,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                 }
                 mma_commit(bar.c_full);
                 SVDC_TRACE_MARK(t3);
-                if (!mbar_wait(bar.a_full, ui & 1u, abort_flag)) { record_timeout(p); goto done; }
+                if (!mbar_wait(bar.a_full, ui & 1u, abort_flag, 11)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
                 SVDC_TRACE_ADD(3, t3);
                 tc_fence_after();
                 for (int g = 0; g < G; ++g, ++iv, ++ig) {           // pass 2: acc = C (V slice)^T
@@ -553,11 +578,18 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                     const int nsub = min(p.gc, CT - cg);
                     const uint32_t vs = iv % p.v_slots, as = ig % p.acc_stages;
                     SVDC_TRACE_MARK(t4);
-                    if (!mbar_wait(bar.v_full + 8 * vs, (iv / p.v_slots) & 1u, abort_flag)) { record_timeout(p); goto done; }
+                    if (!mbar_wait(bar.v_full + 8 * vs, (iv / p.v_slots) & 1u, abort_flag, 12)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
                     SVDC_TRACE_ADD(4, t4);
                     SVDC_TRACE_MARK(t5);
-                    if (!mbar_wait(bar.acc_empty + 8 * as, ((ig / p.acc_stages) & 1u) ^ 1u, abort_flag)) { record_timeout(p); goto done; }
+                    if (!mbar_wait(bar.acc_empty + 8 * as, ((ig / p.acc_stages) & 1u) ^ 1u, abort_flag, 13)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
                     SVDC_TRACE_ADD(5, t5);
+                    // The MMAs of pass 2 do not read F, but this thread waits for the group's F chunks
+                    // all the same: it must see every phase of a ring slot's barrier, or the wait for
+                    // the slot's next pass-1 chunk could be satisfied by a phase before the skipped one.
+                    for (int j = 0; j < nsub; ++j, ++it) {
+                        const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
+                        if (!mbar_wait(bar.full + 8 * s, ph, abort_flag, 19)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
+                    }
                     tc_fence_after();
                     SVDC_TRACE_MARK(t6);
                     const uint32_t idesc = idesc_bf16(kTileRows, nsub * kTileCols);
@@ -578,7 +610,6 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                     SVDC_TRACE_ADD(6, t6);
                 }
                 mma_commit(p2_done);
-                it += CT;   // pass-2 slots are consumed by the epilogue alone
             }
         }
     } else {
@@ -611,11 +642,11 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                 const bool first = *(volatile uint32_t *)&hdr->full_steps == 0;
                 bool ok = true;
                 SVDC_TRACE_MARK(c0);
-                if (!first) { ok = mbar_wait(chat_full, nchat & 1u, abort_flag); ++nchat; }
+                if (!first) { ok = mbar_wait(chat_full, nchat & 1u, abort_flag, 14); ++nchat; }
                 SVDC_TRACE_ADD(0, c0);
                 SVDC_TRACE_MARK(c1);
-                ok = ok && mbar_wait(bar.c_full, ui & 1u, abort_flag);
-                if (!__all_sync(0xFFFFFFFFu, ok)) { record_timeout(p); goto done; }
+                ok = ok && mbar_wait(bar.c_full, ui & 1u, abort_flag, 15);
+                if (!__all_sync(0xFFFFFFFFu, ok)) { record_timeout(p, abort_flag, it, ig, ui); goto done; }
                 SVDC_TRACE_ADD(1, c1);
                 tc_fence_after();
                 SVDC_TRACE_MARK(c2);
@@ -720,16 +751,17 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                 const int cg = (G - 1 - g) * p.gc;
                 const int nsub = min(p.gc, CT - cg);
                 const uint32_t as = ig % p.acc_stages, aph = (ig / p.acc_stages) & 1u;
+                const int last_own = last_own_chunk(it, nsub, grp);
+                SVDC_TRACE_MARK(e3);
+                if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar.acc_full + 8 * as, aph, abort_flag, 16))) { record_timeout(p, abort_flag, it, ig, ui); goto done; }
+                SVDC_TRACE_ADD(3, e3);
+                if (last_own < 0 && lane == 0) mbar_arrive(bar.acc_empty + 8 * as);
                 for (int j = 0; j < nsub; ++j, ++it) {
                     if ((it & 1u) != grp) continue;
                     const int c = cg + j;
                     const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                    SVDC_TRACE_MARK(e3);
-                    bool ok = mbar_wait(bar.acc_full + 8 * as, aph, abort_flag);
-                    SVDC_TRACE_ADD(3, e3);
                     SVDC_TRACE_MARK(e4);
-                    ok = ok && mbar_wait(bar.full + 8 * s, ph, abort_flag);
-                    if (!__all_sync(0xFFFFFFFFu, ok)) { record_timeout(p); goto done; }
+                    if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar.full + 8 * s, ph, abort_flag, 17))) { record_timeout(p, abort_flag, it, ig, ui); goto done; }
                     SVDC_TRACE_ADD(4, e4);
                     tc_fence_after();
                     SVDC_TRACE_MARK(e5);
@@ -744,7 +776,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                     tmem_wait_ld();
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive_n(bar.acc_empty + 8 * as, j == nsub - 1 ? 1u + (uint32_t)(p.gc - nsub) : 1u);
+                    if (lane == 0 && j == last_own) mbar_arrive(bar.acc_empty + 8 * as);   // this warp is done with the group
 #pragma unroll
                     for (int cc = 0; cc < 8; ++cc)
                         sts128(tile + (((uint32_t)cc) ^ ((uint32_t)row & 7u)) * 16u,
@@ -783,7 +815,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
             // the A region is free: stage the next unit's previous Chat there.
             if (issuer) {
                 const int un_next = u + gridDim.x;
-                const bool ok = mbar_wait(p2_done, ui & 1u, abort_flag);
+                const bool ok = mbar_wait(p2_done, ui & 1u, abort_flag, 18);
                 if (ok && un_next < p.units) {
                     const Unit x = decode_unit(p, un_next);
                     if (*(volatile uint32_t *)&header_of(p, x.b)->full_steps != 0) request_chat(x);
@@ -906,6 +938,7 @@ bool fill_full(const StepArgs &a, UmmaParams &p) {
     if (fixed + 2 * (size_t)kTileBytes > avail) return false;
     p.stages = (int)((avail - fixed) / kTileBytes);
     if (p.stages > kMaxStages) p.stages = kMaxStages;
+    p.stages &= ~1;   // even: a slot then always serves the same epilogue group (chunk parity)
     p.a_bufs = 1;
     return true;
 }
@@ -923,6 +956,7 @@ bool fill_cached(const StepArgs &a, UmmaParams &p) {
     if ((size_t)p.a_bufs * p.a_bytes + fixed + 2 * (size_t)kTileBytes > avail) return false;
     p.stages = (int)((avail - (size_t)p.a_bufs * p.a_bytes - fixed) / kTileBytes);
     if (p.stages > kMaxStages) p.stages = kMaxStages;
+    p.stages &= ~1;   // even: a slot then always serves the same epilogue group (chunk parity)
     return true;
 }
 size_t smem_bytes_cached(const UmmaParams &p) {

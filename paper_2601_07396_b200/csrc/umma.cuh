@@ -87,7 +87,9 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 // the kernel tears down normally with an error recorded for the host.
 constexpr long long kWaitCycles = 4000000000LL;
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+// `site` (> 0) names the call; the first wait of a CTA to run out leaves its site in the
+// abort flag, so the host can be told which wait it was.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int site = 255) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (uint32_t it = 1;; ++it) {
@@ -95,7 +97,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if ((it & 63u) == 0u) {
             if (*abort_flag) return false;
             if (clock64() - t0 > kWaitCycles) {
-                *abort_flag = 1;
+                atomicCAS(const_cast<int *>(abort_flag), 0, site);
                 return false;
             }
         }
