@@ -35,18 +35,20 @@ METRIC = "fused full/cached-step HBM GB/s and % of B200 HBM roofline (FLUX-shape
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel (the
-# batched cached step), from the ncu capture summarised under profiles/ (captured on a
-# smaller block count and scaled by blocks, since traffic is proportional to blocks).
-# None until a capture exists for the workload.
-NCU_TRAFFIC_BYTES_PER_BLOCK = {}
+# dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel (the batched cached
+# step, tcgen05 family), per block, from the ncu capture summarised in
+# profiles/umma_cached_kernel_flux_8blocks.txt: taken on 8 blocks of the same shape and
+# scaled by the block count (traffic is proportional to the blocks a launch covers).  The
+# tail of the output that is still in L2 when the kernel ends is not in the counter.
+NCU_TRAFFIC_BYTES_PER_BLOCK = {("flux", 2): 51907520}
 
 
 def algorithmic_bytes(spec: streams.StreamSpec, nblocks: int):
-    """Bytes the method must move per launch: F in / R out (full), R in / Fhat out
-    (cached), the fp32 coefficient arrays, and the basis once per block."""
+    """Bytes the method must move per launch.  Full step: F in, R out, Chat read and written,
+    its split-bf16 operand copy written (3 N k fp32-sized arrays), the basis once.  Cached
+    step: R in, Fhat out, the operand copy of Chat in, the basis once."""
     N, D, k, b = spec.rows, spec.D, spec.k, spec.elem_bytes
-    full = 2 * N * D * b + 2 * N * k * 4 + 2 * D * k * b     # Chat read + write (C_out not requested); V and V^T
+    full = 2 * N * D * b + 3 * N * k * 4 + D * k * b
     cached = 2 * N * D * b + N * k * 4 + D * k * b
     return full * nblocks, cached * nblocks
 
