@@ -56,6 +56,7 @@ extern "C" {
 #define SVDCACHE_ERR_TIMEOUT      (-6) /* a bounded in-kernel wait ran out              */
 #define SVDCACHE_ERR_CUDA         (-7) /* a CUDA runtime / driver call failed           */
 #define SVDCACHE_ERR_NOT_CONVERGED (-8) /* eigen-solver hit its iteration limit         */
+#define SVDCACHE_ERR_SCRATCH_LIMIT (-9) /* problem needs more than the built-in scratch    */
 
 #define SVDCACHE_F32   0
 #define SVDCACHE_BF16  1
@@ -102,6 +103,38 @@ SVDCACHE_API int svdcache_calibrate_finish(int D, int k, float *Vk, double *lamb
 SVDCACHE_API int svdcache_calibrate(const void *Fstack, int64_t M, int D, int64_t ld, int dtype, int k,
                        float *Vk, double *lambda, double *trace, double *info,
                        void *workspace, size_t workspace_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------------
+ * Calibration for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this entry point exists for how the library gets embedded, not for the
+ * method.)
+ *
+ * svdcache_calibrate wants a workspace, and a host program normally gets one from
+ * cudaMalloc.  Some hosts may not call it where calibration has to run: a plugin inside
+ * an inference server whose memory pool was sized and handed out at start-up, code that
+ * runs between the launches of a latency-critical loop where an allocation would
+ * synchronise the device, or a process whose allocator is simply owned by someone else.
+ * For them the library carries SVDCACHE_BUILTIN_SCRATCH_BYTES of scratch inside its own
+ * device image (every GPU that loads the library holds that much until the process exits)
+ * and this call uses it in place of the workspace.  Same arguments, results and status
+ * codes as svdcache_calibrate otherwise; inputs and outputs are still the caller's.
+ *
+ *   - Size limit: svdcache_calibrate_workspace_bytes(D, k) must not exceed
+ *     SVDCACHE_BUILTIN_SCRATCH_BYTES (e.g. D = 512 with k = 64 fits, D = 1152 does not);
+ *     beyond it the call returns SVDCACHE_ERR_SCRATCH_LIMIT and launches nothing.
+ *   - It calls no cudaMalloc / cudaFree and no routine that allocates.
+ *   - The first call on a device looks up the scratch's device address
+ *     (cudaGetSymbolAddress, with that device current) and keeps it; make that first call
+ *     before starting any stream capture.
+ *   - There is ONE scratch array per device and every call uses it.  It still holds the
+ *     previous call's contents when a call starts; the call clears what it accumulates into
+ *     before use.  Two calls whose GPU work overlaps (different streams, different threads)
+ *     would trample each other: keep them ordered, e.g. on one stream.
+ *   - Like svdcache_calibrate it synchronises `stream` while it iterates.
+ * ------------------------------------------------------------------------------- */
+#define SVDCACHE_BUILTIN_SCRATCH_BYTES (4u << 20)
+SVDCACHE_API int svdcache_calibrate_noalloc(const void *Fstack, int64_t M, int D, int64_t ld, int dtype, int k,
+                               float *Vk, double *lambda, double *trace, double *info, void *stream);
 
 /* Rank selection by energy threshold (Eq. 6): the smallest k' <= n with
  * sum_{i<=k'} lambda_i / trace >= tau; n if the n listed eigenvalues fall short.

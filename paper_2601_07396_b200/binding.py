@@ -32,6 +32,7 @@ SIGNATURES = {
     "svdcache_calibrate_accumulate": (_ci, [_vp, _i64, _ci, _i64, _ci, _vp, _sz, _vp]),
     "svdcache_calibrate_finish": (_ci, [_ci, _ci, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "svdcache_calibrate": (_ci, [_vp, _i64, _ci, _i64, _ci, _ci, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "svdcache_calibrate_noalloc": (_ci, [_vp, _i64, _ci, _i64, _ci, _ci, _vp, _vp, _vp, _vp, _vp]),
     "svdcache_rank_for_energy": (_ci, [_vp, _ci, ctypes.c_double, ctypes.c_double, ctypes.POINTER(_ci)]),
     "svdcache_basis_bytes": (_ci, [_ci, _ci, _ci, _szp]),
     "svdcache_basis_layout": (_ci, [_ci, _ci, _ci, _szp, _szp, _szp, _szp]),
@@ -185,6 +186,25 @@ def svdcache_calibrate(Fstack: torch.Tensor, k: int, workspace: Optional[torch.T
     if rc != 0 and (strict or rc != -8):
         raise SvdCacheError(rc, "calibrate")
     return Vk, lam, tr, list(info)
+
+
+BUILTIN_SCRATCH_BYTES = 4 << 20
+
+
+def svdcache_calibrate_noalloc(Fstack: torch.Tensor, k: int, Vk: torch.Tensor, lam: torch.Tensor,
+                               tr: torch.Tensor, stream=None, strict: bool = True):
+    """Calibration on the library's built-in scratch, for callers that may not allocate
+    device memory: the outputs (Vk [D x k] fp32, lam [k] fp64, tr [1] fp64) are passed in,
+    and neither this wrapper nor the call behind it allocates anything on the device.
+    Returns the info list."""
+    M, D = Fstack.shape
+    assert Fstack.stride(1) == 1 and Vk.shape == (D, k) and Vk.dtype == torch.float32 and Vk.is_contiguous()
+    info = (ctypes.c_double * 4)()
+    rc = lib().svdcache_calibrate_noalloc(_ptr(Fstack), M, D, Fstack.stride(0), _dt(Fstack), k, _ptr(Vk),
+                                          _ptr(lam), _ptr(tr), ctypes.cast(info, _vp), _stream(stream))
+    if rc != 0 and (strict or rc != -8):
+        raise SvdCacheError(rc, "calibrate_noalloc")
+    return list(info)
 
 
 def svdcache_rank_for_energy(lam, trace: float, tau: float) -> int:

@@ -78,6 +78,7 @@ const char *svdcache_status_string(int status) {
         case SVDCACHE_ERR_TIMEOUT: return "a bounded in-kernel wait ran out";
         case SVDCACHE_ERR_CUDA: return "CUDA call failed";
         case SVDCACHE_ERR_NOT_CONVERGED: return "eigen-solver did not converge";
+        case SVDCACHE_ERR_SCRATCH_LIMIT: return "problem needs more scratch than the library carries built in";
         default: return "unknown status";
     }
 }

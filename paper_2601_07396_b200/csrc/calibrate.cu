@@ -12,6 +12,7 @@
 // anywhere in this path would miss a 1e-4 bound on the principal-angle cosines.
 #include <algorithm>
 #include <cmath>
+#include <mutex>
 #include <utility>
 
 #include "internal.cuh"
@@ -605,3 +606,61 @@ int calib_finish(int D, int k, float *Vk, double *lambda, double *trace, double 
 }
 
 }  // namespace svdc
+
+// ---------------------------------------------------------------------------------------
+// Calibration without a caller-supplied workspace: the scratch that carries G and the
+// iteration blocks is a fixed array in the library's own device image.
+// ---------------------------------------------------------------------------------------
+namespace svdc {
+namespace {
+
+constexpr size_t kBuiltinScratchBytes = SVDCACHE_BUILTIN_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_builtin_scratch[kBuiltinScratchBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void *g_scratch_addr[kMaxDevices] = {};   // device address of g_builtin_scratch, per device ordinal
+
+// In host code `g_builtin_scratch` only names the symbol; the address a kernel can use
+// has to be asked for, once per device, with that device current.
+int builtin_scratch(void **out) {
+    int dev = -1;
+    int rc = record_cuda(cudaGetDevice(&dev));
+    if (rc) return rc;
+    if (dev < 0 || dev >= kMaxDevices) return SVDCACHE_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_scratch_addr[dev]) {
+        void *ptr = nullptr;
+        rc = record_cuda(cudaGetSymbolAddress(&ptr, g_builtin_scratch));
+        if (rc) return rc;
+        g_scratch_addr[dev] = ptr;
+    }
+    *out = g_scratch_addr[dev];
+    return SVDCACHE_OK;
+}
+
+}  // namespace
+}  // namespace svdc
+
+extern "C" int svdcache_calibrate_noalloc(const void *Fstack, int64_t M, int D, int64_t ld, int dtype, int k,
+                                          float *Vk, double *lambda, double *trace, double *info, void *stream) {
+    using namespace svdc;
+    if (dtype != SVDCACHE_F32 && dtype != SVDCACHE_BF16) return SVDCACHE_ERR_INVALID_ARG;
+    if (M < 1 || D < 8 || D > 16384 || (D % 8) != 0) return SVDCACHE_ERR_BAD_SHAPE;
+    if (k < 8 || k > 256 || (k % 8) != 0 || k > D) return SVDCACHE_ERR_BAD_SHAPE;
+    if (!Fstack || !Vk) return SVDCACHE_ERR_INVALID_ARG;
+    if (ld < D) return SVDCACHE_ERR_BAD_SHAPE;
+    if (((size_t)ld * elem_bytes(dtype)) % 16 != 0) return SVDCACHE_ERR_BAD_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(Fstack) & 15u) || (reinterpret_cast<uintptr_t>(Vk) & 15u)) return SVDCACHE_ERR_BAD_ALIGN;
+    if (calib_workspace_bytes(D, k) > kBuiltinScratchBytes) return SVDCACHE_ERR_SCRATCH_LIMIT;
+    void *ws = nullptr;
+    int rc = builtin_scratch(&ws);
+    if (rc) return rc;
+    cudaStream_t s = (cudaStream_t)stream;
+    rc = calib_begin(D, k, ws, s);   // clears the header and G: nothing of the previous call is reused
+    if (rc) return rc;
+    rc = calib_accumulate(Fstack, M, D, ld, dtype, ws, s);
+    if (rc) return rc;
+    return calib_finish(D, k, Vk, lambda, trace, info, ws, s);
+}
+
