@@ -90,7 +90,15 @@ SVDCACHE_API const char *svdcache_last_cuda_error(void);
  * begin and accumulate only enqueue work.  finish synchronises `stream` several times
  * (it reads convergence numbers back) and returns SVDCACHE_ERR_NOT_CONVERGED if the
  * residual target was not met within the iteration limit (outputs are still written).
- * G is accumulated in fp64 in a fixed order: results are bit-reproducible run to run.
+ * G is accumulated in a fixed order: results are bit-reproducible run to run.  fp32 stacks,
+ * narrow or short bf16 stacks are summed in fp64 throughout (eigenvalues good to ~1e-10
+ * relative).  bf16 stacks of at least 2048 rows per accumulate call whose width is a
+ * multiple of 128 go through the tensor cores: exact bf16 products, fp32 sums over chunks of
+ * 2048 rows, fp64 across chunks.  The tensor cores truncate the fp32 running sum, so G comes
+ * out smaller by a few 1e-6, almost uniformly: eigenvalues (and the trace) carry that
+ * relative error, the eigenvectors are affected far below the 1e-4 principal-angle bound.
+ * Chunks start at the first row of each accumulate call, so feeding the same stack in
+ * different pieces changes the last bits on that path.
  * ------------------------------------------------------------------------------- */
 SVDCACHE_API int svdcache_calibrate_workspace_bytes(int D, int k, size_t *bytes /* host, out */);
 SVDCACHE_API int svdcache_calibrate_begin(int D, int k, void *workspace, size_t workspace_bytes, void *stream);

@@ -19,16 +19,16 @@
 
 namespace svdc {
 
+// tensor-core Gram (gram_umma.cu)
 bool umma_gram_supported(int64_t M, int D, int64_t ld, int dtype);
-int umma_gram_accumulate(const void *F, int64_t M, int D, int64_t ld, double *G, void *scratch,
-                         size_t scratch_bytes, cudaStream_t s);
-size_t umma_gram_scratch_bytes(int D);
+int umma_gram_accumulate(const void *F, int64_t M, int D, int64_t ld, double *G, int *status, cudaStream_t s);
 
 namespace {
 
 struct CalibHeader {
     int32_t D, k_max;
     int64_t rows;
+    int32_t status;   // SVDCACHE_OK, or the error a kernel of the accumulation recorded
 };
 
 int ritz_width(int D, int k) {
@@ -38,7 +38,7 @@ int ritz_width(int D, int k) {
 }
 
 struct CalibLayout {
-    size_t G, Q, Z, T, S, W, X, theta, resid, scal, dead, gram_scratch, total;
+    size_t G, Q, Z, T, S, W, X, theta, resid, scal, dead, total;
     int m;
 };
 
@@ -58,7 +58,6 @@ CalibLayout calib_layout(int D, int k) {
     L.resid = at; at += align_up((size_t)L.m * 8, kAlign);
     L.scal = at; at += kAlign;
     L.dead = at; at += align_up((size_t)L.m * 4, kAlign);
-    L.gram_scratch = at; at += umma_gram_scratch_bytes(D);
     L.total = at;
     return L;
 }
@@ -165,7 +164,7 @@ __global__ void zero_kernel(double *p, int64_t n) {
 }
 
 __global__ void init_header_kernel(CalibHeader *h, int D, int k) {
-    h->D = D; h->k_max = k; h->rows = 0;
+    h->D = D; h->k_max = k; h->rows = 0; h->status = SVDCACHE_OK;
 }
 
 __global__ void add_rows_kernel(CalibHeader *h, int64_t M) { h->rows += M; }
@@ -465,8 +464,7 @@ int calib_accumulate(const void *F, int64_t M, int D, int64_t ld, int dtype, voi
     double *G = (double *)(w + kHeaderBytes);
     int rc;
     if (umma_gram_supported(M, D, ld, dtype)) {
-        const CalibLayout L = calib_layout(D, 8);
-        rc = umma_gram_accumulate(F, M, D, ld, G, w + L.gram_scratch, umma_gram_scratch_bytes(D), s);
+        rc = umma_gram_accumulate(F, M, D, ld, G, &reinterpret_cast<CalibHeader *>(w)->status, s);
     } else if (dtype == SVDCACHE_BF16) {
         const __nv_bfloat16 *f = (const __nv_bfloat16 *)F;
         rc = dgemm<__nv_bfloat16, __nv_bfloat16, true>(f, ld, f, ld, G, D, D, D, M, true, true, s);
@@ -526,6 +524,16 @@ int calib_finish(int D, int k, float *Vk, double *lambda, double *trace, double 
     count_launch(3);
     int rc = check_last_launch();
     if (rc) return rc;
+
+    // an accumulation kernel whose bounded wait ran out has left its error in the header
+    {
+        CalibHeader h;
+        rc = record_cuda(cudaMemcpyAsync(&h, w, sizeof(h), cudaMemcpyDeviceToHost, s));
+        if (rc) return rc;
+        rc = record_cuda(cudaStreamSynchronize(s));
+        if (rc) return rc;
+        if (h.status != SVDCACHE_OK) return h.status;
+    }
 
     int *dead = (int *)(w + L.dead);
     double *Q = nullptr;

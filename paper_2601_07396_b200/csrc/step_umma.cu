@@ -1076,10 +1076,4 @@ int umma_full_step(const StepArgs &a, cudaStream_t s) {
     return check_last_launch();
 }
 
-bool umma_gram_supported(int64_t, int, int64_t, int) { return false; }
-size_t umma_gram_scratch_bytes(int) { return 0; }
-int umma_gram_accumulate(const void *, int64_t, int, int64_t, double *, void *, size_t, cudaStream_t) {
-    return SVDCACHE_ERR_BAD_SHAPE;
-}
-
 }  // namespace svdc
