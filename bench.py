@@ -117,12 +117,26 @@ def dist_env():
 
 
 def reduce_max(value: float, world: int, device) -> float:
+    """Max over ranks of a per-rank number (the timed region's duration)."""
     if world == 1:
         return value
     import torch.distributed as dist
     t = torch.tensor([value], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
+
+
+def rank_blocks(spec, rank: int, nblocks: int):
+    """Blocks of the stream that rank `rank` owns: every rank gets `nblocks` blocks of its
+    own (block ids rank * spec.blocks + 0 ..), so ranks never share a block and the step
+    kernels need no collective (weak scaling)."""
+    first = rank * spec.blocks
+    return list(range(first, first + nblocks))
+
+
+def whole_job_value(step_bytes: int, steps: int, world: int, max_ms: float) -> float:
+    """GB/s of the whole job: bytes all ranks processed / the slowest rank's time."""
+    return world * step_bytes * steps / (max_ms * 1e-3) / 1e9
 
 
 # ------------------------------------------------------------------------- ours ---
@@ -172,7 +186,7 @@ def run_ours(args):
 
     spec = streams.SPECS[args.workload]
     nblocks = args.blocks or (spec.blocks if spec.name != "hunyuan" else 8)
-    wl = build_workload(spec, nblocks, device, block_offset=rank * spec.blocks)
+    wl = build_workload(spec, nblocks, device, block_offset=rank_blocks(spec, rank, nblocks)[0])
     F, bases, state, Fhat, dt = wl["F"], wl["bases"], wl["state"], wl["Fhat"], wl["dt"]
     k, beta, interval = spec.k, spec.beta, spec.interval
     bytes_full, bytes_cached = algorithmic_bytes(spec, nblocks)
@@ -246,8 +260,8 @@ def run_ours(args):
     if rank != 0:
         return
     peak, peak_kind = measured_peak()
-    value = world * step_bytes * args.steps / (total_ms * 1e-3) / 1e9
-    e2e_value = world * step_bytes * e2e_steps / (e2e_ms * 1e-3) / 1e9
+    value = whole_job_value(step_bytes, args.steps, world, total_ms)
+    e2e_value = whole_job_value(step_bytes, e2e_steps, world, e2e_ms)
     cached_avg_ms = sum(cached_ms) / max(1, len(cached_ms))
     full_avg_ms = sum(full_ms) / max(1, len(full_ms))
     cached_gbs = bytes_cached / (cached_avg_ms * 1e-3) / 1e9 if cached_ms else None
@@ -367,6 +381,91 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def run_sweep(args):
+    """Rank and calibration sweep on the FLUX shape: one JSON line per rank k (both fused
+    step kernels, batched over `--blocks` blocks) and per calibration stack size M (Gram on
+    the tensor cores, then the eigen-solver).  One GPU; not the headline line."""
+    from paper_2601_07396_b200 import binding as sc
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    peak, peak_kind = measured_peak()
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
+            tf_peak = float(json.load(fh)["bf16_tflops"])
+    except Exception:
+        tf_peak = 1590.0
+    base = streams.FLUX
+    nb = args.blocks or 16
+    N, D = base.rows, base.D
+
+    def timed(fn, reps):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    F = torch.empty(nb, N, D, dtype=torch.bfloat16, device=device)
+    for b in range(nb):
+        streams.BlockStream(base, b, device=device).features(0, out=F[b])
+    Fhat = torch.empty_like(F)
+    V_gen = streams.BlockStream(base, 0, device=device).V_gen     # D x 256, orthonormal
+    for k in streams.SWEEP_RANKS:
+        spec = streams.StreamSpec(**{**base.__dict__, "k": k})
+        Vk = V_gen[:, :k].float().contiguous()
+        bases = torch.empty(nb, sc.svdcache_basis_bytes(D, k, sc.BF16), dtype=torch.uint8, device=device)
+        for b in range(nb):
+            sc.svdcache_basis_prepare(Vk, sc.BF16, basis=bases[b])
+        state = sc.new_state(N, D, k, sc.BF16, device, blocks=nb)
+        bf, bc = algorithmic_bytes(spec, nb)
+        ms_f = timed(lambda: sc.svdcache_full_step_batched(F, bases, state, k, spec.beta), args.steps)
+        ms_c = timed(lambda: sc.svdcache_cached_step_batched(state, bases, Fhat, k), args.steps)
+        gf, gc = bf / ms_f / 1e6, bc / ms_c / 1e6
+        # split-bf16 operand: 2 N D k flops in pass 1, 4 N D k in pass 2 / the cached product
+        tf_f, tf_c = nb * 6.0 * N * D * k / ms_f / 1e9, nb * 4.0 * N * D * k / ms_c / 1e9
+        print(json.dumps({"sweep": "rank", "k": k, "blocks": nb, "rows": N, "D": D,
+                          "full_step": {"ms": round(ms_f, 4), "GBps": round(gf, 1), "frac_hbm": round(gf / peak, 4),
+                                        "TFLOPs": round(tf_f, 1), "frac_tensor": round(tf_f / tf_peak, 4)},
+                          "cached_step": {"ms": round(ms_c, 4), "GBps": round(gc, 1), "frac_hbm": round(gc / peak, 4),
+                                          "TFLOPs": round(tf_c, 1), "frac_tensor": round(tf_c / tf_peak, 4)},
+                          "peaks": {"hbm_GBps": peak, "bf16_TFLOPs": tf_peak, "source": peak_kind}}), flush=True)
+        del state, bases
+    del F, Fhat
+    torch.cuda.empty_cache()
+    k = base.k
+    for M in streams.SWEEP_CALIB_ROWS:
+        snaps = max(1, M // N)
+        stack = streams.calibration_stack(base, 0, device=device,
+                                          trajectories=tuple(range(1, 1 + (snaps + 7) // 8)),
+                                          timesteps=base.calib_timesteps[:min(8, snaps)])[:M]
+        ws = torch.empty(sc.svdcache_calibrate_workspace_bytes(D, k), dtype=torch.uint8, device=device)
+
+        def gram():
+            sc.svdcache_calibrate_begin(D, k, ws)
+            sc.svdcache_calibrate_accumulate(stack, ws)
+        ms_g = timed(gram, 3)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        Vk, lam, tr, info = sc.svdcache_calibrate_finish(D, k, ws, strict=False)
+        e1.record()
+        torch.cuda.synchronize()
+        tf = 2.0 * M * D * D / ms_g / 1e9
+        print(json.dumps({"sweep": "calibration", "M": int(stack.shape[0]), "D": D, "k": k,
+                          "gram": {"ms": round(ms_g, 3), "TFLOPs_full_square": round(tf, 1),
+                                   "frac_tensor": round(tf / tf_peak, 4),
+                                   "note": "2 M D^2 flops counted; the upper block triangle computed is 156/288 of that"},
+                          "eigen": {"ms": round(e0.elapsed_time(e1), 1), "multiplications_by_G": info[0],
+                                    "max_rel_residual": info[1]}}), flush=True)
+        del stack, ws
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -379,10 +478,13 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--ref-rows", type=int, default=1024)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="rank and calibration sweep on the FLUX shape")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
