@@ -231,8 +231,12 @@ SVDCACHE_API int svdcache_cached_step_batched(int nblocks, const void *state, si
  *   svdcache_kernel_launches: kernels this library has launched in this process.
  *   svdcache_set_path: 0 = pick automatically, 1 = force the CUDA-core kernels,
  *                      2 = force the tcgen05 kernels (error if the shape is outside
- *                      what they support).  Returns the previous setting.
- *   svdcache_last_path: which kernel family the last step call used (1 or 2).
+ *                      what they support), 3 = as 2, and the full step shares each
+ *                      128-row tile between the two CTAs of a thread-block cluster
+ *                      (each streams half of the columns; the partial coefficients
+ *                      meet through distributed shared memory) where the shape
+ *                      allows it.  Returns the previous setting.
+ *   svdcache_last_path: which kernel family the last step call used (1, 2 or 3).
  * ------------------------------------------------------------------------------- */
 SVDCACHE_API uint64_t svdcache_kernel_launches(void);
 SVDCACHE_API int svdcache_set_path(int path);

@@ -37,12 +37,14 @@ static int check_pitch(int64_t ld, int D, int dtype) {
     return SVDCACHE_OK;
 }
 
-static int dispatch(const StepArgs &a, bool full, cudaStream_t s) {
+static int dispatch(const StepArgs &a_in, bool full, cudaStream_t s) {
+    StepArgs a = a_in;
     const int want = g_path.load();
     const bool can_umma = umma_supported(a, full);
-    if (want == 2 && !can_umma) return SVDCACHE_ERR_BAD_SHAPE;
-    const bool use_umma = (want == 2) || (want == 0 && can_umma);
-    g_last_path.store(use_umma ? 2 : 1);
+    if (want >= 2 && !can_umma) return SVDCACHE_ERR_BAD_SHAPE;
+    const bool use_umma = (want >= 2) || (want == 0 && can_umma);
+    a.cluster_split = (want == 3) ? 1 : 0;
+    g_last_path.store(use_umma ? (want == 3 ? 3 : 2) : 1);
     if (use_umma) return full ? umma_full_step(a, s) : umma_cached_step(a, s);
     return full ? simt_full_step(a, s) : simt_cached_step(a, s);
 }
@@ -87,7 +89,7 @@ const char *svdcache_last_cuda_error(void) { return g_cuda_error; }
 
 uint64_t svdcache_kernel_launches(void) { return g_launches.load(); }
 int svdcache_set_path(int path) {
-    if (path < 0 || path > 2) return SVDCACHE_ERR_INVALID_ARG;
+    if (path < 0 || path > 3) return SVDCACHE_ERR_INVALID_ARG;
     return g_path.exchange(path);
 }
 int svdcache_last_path(void) { return g_last_path.load(); }

@@ -84,6 +84,7 @@ struct StepArgs {
     int64_t N;
     int D, k, dtype, nblocks;
     float beta;
+    int cluster_split;      // full step, tcgen05 family: share each row tile between the two CTAs of a cluster
 };
 
 // launch bookkeeping (api.cu)

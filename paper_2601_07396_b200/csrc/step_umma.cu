@@ -41,7 +41,8 @@ struct UmmaParams {
     uint32_t a_half_bytes, a_bytes;
     int gc, acc_stages, acc_cols, v_slots;   // chunks per MMA group, TMEM ring, basis ring
     uint32_t vslice_bytes;
-    uint32_t a_region_bytes, chat_stage_off; // full step: A operand (+ Chat staging when k < 64)
+    uint32_t a_region_bytes, chat_stage_off; // full step: A operand (+ Chat staging when it is not in place)
+    int cluster;                             // full step: CTAs that share a row tile (1, or 2 splitting D)
     char *state;
     size_t state_stride, chat_off, ophi_off, oplo_off;
     float *C_out;
@@ -419,6 +420,7 @@ __device__ __forceinline__ void pack_split8(const float *v, uint4 &hi, uint4 &lo
     lo = make_uint4(l[0], l[1], l[2], l[3]);
 }
 
+template <bool kClusterSplit>
 __global__ void __launch_bounds__(kThreadsFull, 1)
 umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant__ CUtensorMap tm_vt,
                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_rout,
@@ -433,7 +435,9 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
     // barriers beyond the ring ones: c_full (C accumulated), a_full (A operand written),
     // p2_done (pass-2 MMAs of the unit finished: the A region may be restaged), chat_full
     // (previous Chat staged)
-    const uint32_t chat_full = bar.a_full + 8, p2_done = bar.c_done;
+    // cluster mode: peer_ready (the peer's A region may be written), recv_full (the peer's
+    // partial C has arrived in mine)
+    const uint32_t chat_full = bar.a_full + 8, p2_done = bar.c_done, peer_ready = bar.a_empty, recv_full = bar.a_empty + 8;
     uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
     volatile int *abort_flag = reinterpret_cast<volatile int *>(gen_base + (bar.abort_flag - base));
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(gen_base + (bar.tmem_slot - base));
@@ -442,18 +446,31 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
     SVDC_TRACE_DECL
     const uint32_t tmem_cols = 512;
     const int CT = p.chunks_total;
-    const int G = (CT + p.gc - 1) / p.gc;               // groups per pass
+    // A cluster of two CTAs shares each row tile: rank r takes a contiguous range of the
+    // column groups in both passes, the partial C's meet through distributed shared memory.
+    constexpr uint32_t csize = kClusterSplit ? 2u : 1u;
+    const uint32_t crank = kClusterSplit ? cluster_ctarank() : 0u;
+    const int cid = (int)(blockIdx.x / csize), nclusters = (int)(gridDim.x / csize);
+    const int G_all = (CT + p.gc - 1) / p.gc;           // groups per pass, whole width
+    const int g_off = (int)((crank * (uint32_t)G_all) / csize);
+    const int G = (int)(((crank + 1u) * (uint32_t)G_all) / csize) - g_off;   // this CTA's groups per pass
+    const int c_first = g_off * p.gc;
+    const int CTm = min(CT, (g_off + G) * p.gc) - c_first;                   // this CTA's chunks per pass
     const uint32_t a_part = p.k >= 64 ? kBlk32Bytes : p.a_half_bytes;   // hi -> lo distance
     const uint32_t a_kb = 2u * kBlk32Bytes;                             // K-block distance (k >= 64)
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < p.stages; ++s) { mbar_init(bar.full + 8 * s, 1); mbar_init(bar.empty + 8 * s, 4); }
+        // F slot: free again after five arrivals -- pass 1: the MMAs' commit plus four from the
+        // MMA thread; pass 2: the four slab stores plus the MMA thread's "seen" (see there)
+        for (int s = 0; s < p.stages; ++s) { mbar_init(bar.full + 8 * s, 1); mbar_init(bar.empty + 8 * s, 5); }
         for (int s = 0; s < p.acc_stages; ++s) { mbar_init(bar.acc_full + 8 * s, 1); mbar_init(bar.acc_empty + 8 * s, 8); }
         for (int s = 0; s < p.v_slots; ++s) { mbar_init(bar.v_full + 8 * s, 1); mbar_init(bar.v_empty + 8 * s, 1); }
         mbar_init(bar.a_full, 128);
         mbar_init(chat_full, 1);
         mbar_init(bar.c_full, 1);
         mbar_init(p2_done, 1);
+        mbar_init(peer_ready, 1);
+        mbar_init(recv_full, 128);
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&tm_f);
@@ -468,6 +485,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
     }
     tc_fence_before();
     __syncthreads();
+    if (csize > 1) cluster_sync_all();   // the peer's barriers exist before anyone arrives on them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
@@ -481,10 +499,10 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
             // other way round -- so the thread polls both rings without blocking.
             struct Step { int u, pass, g; };
             auto next_step = [&](Step x) {
-                if (++x.g == G) { x.g = 0; if (++x.pass == 2) { x.pass = 0; x.u += gridDim.x; } }
+                if (++x.g == G) { x.g = 0; if (++x.pass == 2) { x.pass = 0; x.u += nclusters; } }
                 return x;
             };
-            Step vcur{(int)blockIdx.x, 0, 0}, fcur{(int)blockIdx.x, 0, 0};
+            Step vcur{cid, 0, 0}, fcur{cid, 0, 0};
             uint32_t iv = 0, it = 0;   // basis slices, F chunks requested so far
             int fc = 0;                // next chunk of fcur's group (offset within the group)
             long long t_idle = clock64();
@@ -495,7 +513,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                     const uint32_t vs = iv % p.v_slots;
                     if (mbar_test_wait(bar.v_empty + 8 * vs, ((iv / p.v_slots) & 1u) ^ 1u)) {
                         const Unit un = decode_unit(p, vcur.u);
-                        const int cg = (vcur.pass == 0 ? vcur.g : G - 1 - vcur.g) * p.gc;
+                        const int cg = (g_off + (vcur.pass == 0 ? vcur.g : G - 1 - vcur.g)) * p.gc;
                         const uint32_t vdst = v_base0 + vs * p.vslice_bytes;
                         mbar_arrive_expect_tx(bar.v_full + 8 * vs, p.vslice_bytes);
                         if (vcur.pass == 0) {   // V_k^T columns of each chunk: gc boxes of k rows x 64
@@ -515,7 +533,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                     const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
                     if (mbar_test_wait(bar.empty + 8 * s, ph ^ 1u)) {
                         const Unit un = decode_unit(p, fcur.u);
-                        const int cg = (fcur.pass == 0 ? fcur.g : G - 1 - fcur.g) * p.gc;
+                        const int cg = (g_off + (fcur.pass == 0 ? fcur.g : G - 1 - fcur.g)) * p.gc;
                         const int nsub = min(p.gc, CT - cg);
                         mbar_arrive_expect_tx(bar.full + 8 * s, kTileBytes);
                         tma_load_3d_hint(stage0 + s * kTileBytes, &tm_f, bar.full + 8 * s, (cg + fc) * kTileCols,
@@ -542,10 +560,10 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
             const uint32_t idesc1 = idesc_bf16(kTileRows, p.k);
             const int ksteps = p.kb_elems / 16;
             const uint64_t a_desc0 = smem_desc_kmajor(a_base, p.kb_bytes);
-            for (int u = blockIdx.x; u < p.units; u += gridDim.x, ++ui) {
+            for (int u = cid; u < p.units; u += nclusters, ++ui) {
                 // C of the previous unit has been read out of TMEM: a_full(ui - 1) was awaited below
                 for (int g = 0; g < G; ++g, ++iv) {                 // pass 1: C_a += F_chunk (V^T chunk)^T
-                    const int cg = g * p.gc, ce = min(cg + p.gc, CT);
+                    const int cg = (g_off + g) * p.gc, ce = min(cg + p.gc, CT);
                     const uint32_t vs = iv % p.v_slots;
                     SVDC_TRACE_MARK(t0);
                     if (!mbar_wait(bar.v_full + 8 * vs, (iv / p.v_slots) & 1u, abort_flag, 9)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
@@ -561,9 +579,9 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                         const uint64_t vd = smem_desc_kmajor(v_base0 + vs * p.vslice_bytes + (c - cg) * (p.k * 128), 128);
 #pragma unroll
                         for (int ks = 0; ks < kTileCols / 16; ++ks)
-                            mma_bf16_ss(tmem_base, fd + 2 * ks, vd + 2 * ks, idesc1, (c | ks) != 0 ? 1u : 0u);
+                            mma_bf16_ss(tmem_base, fd + 2 * ks, vd + 2 * ks, idesc1, (c != c_first || ks != 0) ? 1u : 0u);
                         mma_commit(bar.empty + 8 * s);
-                        mbar_arrive_n(bar.empty + 8 * s, 3);   // pass 1 has no slab stores: their three other arrivals
+                        mbar_arrive_n(bar.empty + 8 * s, 4);   // pass 1 has no slab stores: the other four arrivals
                         SVDC_TRACE_ADD(2, t2);
                     }
                     mma_commit(bar.v_empty + 8 * vs);
@@ -574,7 +592,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                 SVDC_TRACE_ADD(3, t3);
                 tc_fence_after();
                 for (int g = 0; g < G; ++g, ++iv, ++ig) {           // pass 2: acc = C (V slice)^T
-                    const int cg = (G - 1 - g) * p.gc;
+                    const int cg = (g_off + G - 1 - g) * p.gc;
                     const int nsub = min(p.gc, CT - cg);
                     const uint32_t vs = iv % p.v_slots, as = ig % p.acc_stages;
                     SVDC_TRACE_MARK(t4);
@@ -583,13 +601,6 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                     SVDC_TRACE_MARK(t5);
                     if (!mbar_wait(bar.acc_empty + 8 * as, ((ig / p.acc_stages) & 1u) ^ 1u, abort_flag, 13)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
                     SVDC_TRACE_ADD(5, t5);
-                    // The MMAs of pass 2 do not read F, but this thread waits for the group's F chunks
-                    // all the same: it must see every phase of a ring slot's barrier, or the wait for
-                    // the slot's next pass-1 chunk could be satisfied by a phase before the skipped one.
-                    for (int j = 0; j < nsub; ++j, ++it) {
-                        const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                        if (!mbar_wait(bar.full + 8 * s, ph, abort_flag, 19)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
-                    }
                     tc_fence_after();
                     SVDC_TRACE_MARK(t6);
                     const uint32_t idesc = idesc_bf16(kTileRows, nsub * kTileCols);
@@ -608,6 +619,16 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                     mma_commit(bar.v_empty + 8 * vs);
                     mma_commit(bar.acc_full + 8 * as);
                     SVDC_TRACE_ADD(6, t6);
+                    // The MMAs of pass 2 do not read F, but this thread still has to see every phase of
+                    // a ring slot's barrier (or its wait for the slot's next pass-1 chunk could be
+                    // satisfied by the phase before a skipped one), and the slot must not be reused
+                    // before it has: it waits for the group's chunks here, after the MMAs are on their
+                    // way, and its arrival is one of the five that free the slot.
+                    for (int j = 0; j < nsub; ++j, ++it) {
+                        const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
+                        if (!mbar_wait(bar.full + 8 * s, ph, abort_flag, 19)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
+                        mbar_arrive(bar.empty + 8 * s);
+                    }
                 }
                 mma_commit(p2_done);
             }
@@ -630,11 +651,11 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
             for (int b = 0; b < nblk; ++b)
                 tma_load_3d(chat_base + b * kBlk32Bytes, &tm_chat, chat_full, b * 32, x.rt * kTileRows, x.b);
         };
-        if (issuer && (int)blockIdx.x < p.units) {
-            const Unit x = decode_unit(p, blockIdx.x);
+        if (issuer && cid < p.units) {
+            const Unit x = decode_unit(p, cid);
             if (*(volatile uint32_t *)&header_of(p, x.b)->full_steps != 0) request_chat(x);
         }
-        for (int u = blockIdx.x; u < p.units; u += gridDim.x, ++ui) {
+        for (int u = cid; u < p.units; u += nclusters, ++ui) {
             const Unit un = decode_unit(p, u);
             if (c_warp) {
                 // ---- C job: TMEM -> EMA -> Chat, split-bf16 A operand (+ the state's operand copy)
@@ -650,13 +671,38 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                 SVDC_TRACE_ADD(1, c1);
                 tc_fence_after();
                 SVDC_TRACE_MARK(c2);
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+                if constexpr (kClusterSplit) {
+                    // Exchange of the partial C's.  My pass-1 MMAs are complete, hence (the tensor
+                    // pipe runs in order) so are the pass-2 MMAs of my previous unit: my A region
+                    // is free, and I tell the peer so.  Once the peer has said the same, every C
+                    // thread writes its row of my partial into the peer's A region (the layout of
+                    // the staged Chat: 32-column blocks of 128-byte swizzled rows) and arrives on
+                    // the peer's recv_full; my own recv_full then says the peer's partial is here.
+                    const uint32_t peer = crank ^ 1u;
+                    if (issuer) mbar_arrive_remote(mapa_shared(peer_ready, peer));
+                    bool okx = mbar_wait_cluster(peer_ready, ui & 1u, abort_flag, 20);
+                    if (!__all_sync(0xFFFFFFFFu, okx)) { record_timeout(p, abort_flag, it, ig, ui); goto done; }
+                    for (int b = 0; b < nblk; ++b) {
+                        uint32_t tmp[32];
+                        tmem_ld_32x32(taddr + b * 32, tmp);
+                        tmem_wait_ld();
+                        const uint32_t rrow = mapa_shared(a_base + (uint32_t)b * kBlk32Bytes + (uint32_t)row * 128u, peer);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            st_cluster128(rrow + (((uint32_t)i) ^ ((uint32_t)row & 7u)) * 16u,
+                                          make_uint4(tmp[4 * i], tmp[4 * i + 1], tmp[4 * i + 2], tmp[4 * i + 3]));
+                    }
+                    mbar_arrive_remote(mapa_shared(recv_full, peer));
+                    okx = mbar_wait_cluster(recv_full, ui & 1u, abort_flag, 21);
+                    if (!__all_sync(0xFFFFFFFFu, okx)) { record_timeout(p, abort_flag, it, ig, ui); goto done; }
+                }
                 const int64_t n = (int64_t)un.rt * kTileRows + row;
-                const bool row_live = n < p.N;
+                const bool row_live = n < p.N && crank == 0;   // in a cluster, rank 0 writes the coefficient arrays
                 char *st_b = p.state + (size_t)un.b * p.state_stride;
                 float *chat_g = reinterpret_cast<float *>(st_b + p.chat_off) + n * p.k;
                 float *cout_g = p.C_out ? reinterpret_cast<float *>((char *)p.C_out + (size_t)un.b * p.C_stride) + n * p.k
                                         : nullptr;
-                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
                 const int nkb64 = p.k >= 64 ? p.nkb : 1;
                 for (int kb = 0; kb < nkb64; ++kb) {
                     // staged previous Chat of this row: the block holding columns kb*64 .. +31 (A) and
@@ -669,6 +715,10 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                     const int halves = p.k >= 64 ? 2 : 1;
                     float prevB[32];
                     if (!first && halves == 2) load_row32(stB, (uint32_t)row, chat_row_bytes, 32, prevB);
+                    // cluster mode: the peer's partial sits where this row's hi / lo operand rows go
+                    // (the staged Chat has a buffer of its own then); read the lo half's block first
+                    float recvB[kClusterSplit ? 32 : 1];
+                    if constexpr (kClusterSplit) load_row32(lo_row, (uint32_t)row, 128u, 32, recvB);
                     for (int h = 0; h < halves; ++h) {
                         const int col0 = kb * 64 + h * 32;
                         const int ncols = p.k - col0 < 32 ? p.k - col0 : 32;
@@ -679,6 +729,17 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                             tmem_wait_ld();
 #pragma unroll
                             for (int i = 0; i < 32; ++i) cs[i] = __uint_as_float(tmp[i]);
+                        }
+                        if constexpr (kClusterSplit) {   // C = my partial + the peer's (a + b == b + a: both CTAs get the same bits)
+                            if (h == 0) {
+                                float recvA[32];
+                                load_row32(hi_row, (uint32_t)row, 128u, 32, recvA);
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) cs[i] += recvA[i];
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) cs[i] += recvB[i];
+                            }
                         }
                         float ch[32];
                         if (first) {
@@ -735,7 +796,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                 mbar_arrive(bar.a_full);
                 SVDC_TRACE_ADD(2, c2);
                 // count this unit; the last unit of a block to get here counts the full step
-                if (issuer) {
+                if (issuer && crank == 0) {
                     const uint32_t prev = atomicAdd(&hdr->done, 1u);
                     if (prev == (uint32_t)p.row_tiles - 1u) {
                         hdr->done = 0;
@@ -746,9 +807,9 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
             // ---- epilogue duty for this group's chunks of pass 2
             const int slab_row0 = un.rt * kTileRows + q * kSlabRows;
             const bool slab_live = (int64_t)slab_row0 < p.N;
-            it += CT;   // pass-1 slots are consumed by the MMA warp alone
+            it += CTm;   // pass-1 slots are consumed by the MMA warp alone
             for (int g = 0; g < G; ++g, ++ig) {
-                const int cg = (G - 1 - g) * p.gc;
+                const int cg = (g_off + G - 1 - g) * p.gc;
                 const int nsub = min(p.gc, CT - cg);
                 const uint32_t as = ig % p.acc_stages, aph = (ig / p.acc_stages) & 1u;
                 const int last_own = last_own_chunk(it, nsub, grp);
@@ -814,7 +875,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
             // Every accumulator of this unit has been read, so its pass-2 MMAs are complete and
             // the A region is free: stage the next unit's previous Chat there.
             if (issuer) {
-                const int un_next = u + gridDim.x;
+                const int un_next = u + nclusters;
                 const bool ok = mbar_wait(p2_done, ui & 1u, abort_flag, 18);
                 if (ok && un_next < p.units) {
                     const Unit x = decode_unit(p, un_next);
@@ -830,6 +891,7 @@ done:
     SVDC_TRACE_FLUSH(g_trace);
     tc_fence_before();
     __syncthreads();
+    if (csize > 1) cluster_sync_all();   // no CTA leaves while its peer may still reach into it
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, tmem_cols);
@@ -922,16 +984,20 @@ void fill_groups(const StepArgs &a, UmmaParams &p) {
 }
 
 // Full step: shared memory = A operand region (+ Chat staging when k < 64) | basis ring | F ring | barriers.
-bool fill_full(const StepArgs &a, UmmaParams &p) {
+bool fill_full(const StepArgs &a, UmmaParams &p, int cluster = 1) {
     if (!fill_params(a, p)) return false;
+    p.cluster = cluster;
     fill_groups(a, p);
     // TMEM: C in columns [0, k), then the pass-2 ring; at least two ring stages
     while (p.gc > 1 && a.k + 2 * p.gc * kTileCols > 512) --p.gc;
     p.acc_cols = p.gc * kTileCols;
     p.acc_stages = (512 - a.k) / p.acc_cols < kAccStages ? (512 - a.k) / p.acc_cols : kAccStages;
     p.vslice_bytes = (uint32_t)p.gc * kTileCols * a.k * 2;
-    p.chat_stage_off = a.k >= 64 ? 0u : p.a_bytes;
-    p.a_region_bytes = p.a_bytes + (a.k >= 64 ? 0u : (uint32_t)kTileRows * a.k * 4u);
+    // the staged previous Chat shares the A region (converted in place) when k >= 64, unless
+    // the region doubles as the receive buffer of a cluster's exchange
+    const bool in_place = a.k >= 64 && cluster == 1;
+    p.chat_stage_off = in_place ? 0u : p.a_bytes;
+    p.a_region_bytes = p.a_bytes + (in_place ? 0u : (uint32_t)kTileRows * a.k * 4u);
     p.a_region_bytes = (p.a_region_bytes + 1023u) & ~1023u;
     const size_t avail = kSmemBudget - 1024 /*alignment*/ - kBarBytes - 64;
     const size_t fixed = (size_t)p.a_region_bytes + (size_t)p.v_slots * p.vslice_bytes;
@@ -1037,12 +1103,60 @@ int umma_cached_step(const StepArgs &a, cudaStream_t s) {
     return check_last_launch();
 }
 
+// Largest number of 2-CTA clusters of the full-step kernel that can be resident at once.
+int max_full_clusters(size_t smem) {
+    static int cached = -1;
+    if (cached >= 0) return cached;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * num_sms());
+    cfg.blockDim = dim3(kThreadsFull);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, umma_full_kernel<true>, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+    cached = n;
+    return n;
+}
+
 int umma_full_step(const StepArgs &a, cudaStream_t s) {
     UmmaParams p{};
     if (!fill_full(a, p)) return SVDCACHE_ERR_BAD_SHAPE;
     p.dsplit = 1;
     p.chunks_per_slice = p.chunks_total;
     p.units = p.row_tiles * a.nblocks;
+
+    static bool attr_set = false;
+    if (!attr_set) {
+        int rc0 = record_cuda(cudaFuncSetAttribute(umma_full_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   (int)kSmemBudget));
+        if (rc0) return rc0;
+        rc0 = record_cuda(cudaFuncSetAttribute(umma_full_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               (int)kSmemBudget));
+        if (rc0) return rc0;
+        attr_set = true;
+    }
+    // Two CTAs per row tile (each streams half the columns in both passes) halve the F bytes
+    // that must survive in L2 between the passes.  On request only: the exchange of the partial
+    // C's lengthens the serial part of every tile and the F ring is shorter, which today costs
+    // more than the L2 hits bring.  Needs the split operand layout (k >= 64), at least two
+    // column groups and an F ring of six slots.
+    int nclusters = 0;
+    {
+        UmmaParams pc{};
+        const int groups = (p.chunks_total + p.gc - 1) / p.gc;
+        if (a.cluster_split && a.k >= 64 && groups >= 2 && fill_full(a, pc, 2) && pc.stages >= 6) {
+            const int fit = max_full_clusters(smem_bytes_full(pc));
+            if (fit >= num_sms() / 2 - 4) {   // else the cluster placement leaves too many SMs idle
+                pc.dsplit = 1; pc.chunks_per_slice = pc.chunks_total; pc.units = p.units;
+                p = pc;
+                nclusters = p.units < fit ? p.units : fit;
+            }
+        }
+    }
 
     const StateLayout SL = state_layout(a.N, a.D, a.k, a.dtype);
     const BasisLayout BL = basis_layout(a.D, a.k, a.dtype);
@@ -1063,15 +1177,23 @@ int umma_full_step(const StepArgs &a, cudaStream_t s) {
     if (rc) return rc;
 
     const size_t smem = smem_bytes_full(p);
-    static bool attr_set = false;
-    if (!attr_set) {
-        rc = record_cuda(cudaFuncSetAttribute(umma_full_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              (int)kSmemBudget));
-        if (rc) return rc;
-        attr_set = true;
+    if (p.cluster == 2) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * nclusters);
+        cfg.blockDim = dim3(kThreadsFull);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = s;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        rc = record_cuda(cudaLaunchKernelEx(&cfg, umma_full_kernel<true>, tm_f, tm_vt, tm_v, tm_rout, tm_chat, p));
+        count_launch();
+        return rc ? rc : check_last_launch();
     }
     const int grid = p.units < num_sms() ? p.units : num_sms();
-    umma_full_kernel<<<grid, kThreadsFull, smem, s>>>(tm_f, tm_vt, tm_v, tm_rout, tm_chat, p);
+    umma_full_kernel<false><<<grid, kThreadsFull, smem, s>>>(tm_f, tm_vt, tm_v, tm_rout, tm_chat, p);
     count_launch();
     return check_last_launch();
 }

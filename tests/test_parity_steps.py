@@ -120,6 +120,18 @@ def test_shapes_and_ragged_tails(N, D, k, dtype, ld_pad):
     _play(spec, 0, Vk, range(5), ld_pad=ld_pad)
 
 
+@pytest.mark.parametrize("N,D,k", [(300, 1152, 64), (257, 3072, 128), (1000, 512, 64), (129, 3072, 64)])
+def test_cluster_split_full_step(N, D, k):
+    """Path 3: the full step with each row tile shared by the two CTAs of a cluster (partial
+    coefficients exchanged through distributed shared memory), same oracle, same bounds.
+    Shapes it does not apply to (here k = 128: the F ring would get too short) must fall back
+    to the one-CTA kernel silently."""
+    spec = streams.StreamSpec("cluster", blocks=1, rows=N, D=D, dtype="bf16", k=k, T=5, interval=2,
+                              rank=min(D, 2 * k), amp=30.0, power=1.0, noise_std=0.02)
+    _play(spec, 0, None, range(5), path=3)
+    assert sc.svdcache_last_path() in (0, 2, 3)
+
+
 def test_batched_equals_per_block_and_oracle():
     spec = streams.StreamSpec("batch", blocks=3, rows=200, D=512, dtype="bf16", k=64, T=4, interval=2,
                               rank=128, amp=30.0, power=1.0, noise_std=0.02)
