@@ -40,6 +40,7 @@ struct UmmaParams {
     int stages, a_bufs;
     uint32_t a_half_bytes, a_bytes;
     int gc, acc_stages, acc_cols, v_slots;   // chunks per MMA group, TMEM ring, basis ring
+    int dual, acc_stride;                    // cached step: separate hi / lo accumulators; TMEM columns per ring stage
     uint32_t vslice_bytes;
     uint32_t a_region_bytes, chat_stage_off; // full step: A operand (+ Chat staging when it is not in place)
     int cluster;                             // full step: CTAs that share a row tile (1, or 2 splitting D)
@@ -191,6 +192,7 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(gen_base + (bar.tmem_slot - base));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    SVDC_TRACE_DECL
     const uint32_t tmem_cols = 512;
 
     if (threadIdx.x == 0) {
@@ -234,7 +236,9 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
                     u_a += gridDim.x;
                     if (*(volatile uint32_t *)&header_of(p, ux.b)->full_steps == 0) continue;
                     const uint32_t ab = ua % p.a_bufs;
+                    SVDC_TRACE_MARK(p0);
                     if (!mbar_wait(bar.a_empty + 8 * ab, ((ua / p.a_bufs) & 1u) ^ 1u, abort_flag, 1)) { record_timeout(p, abort_flag); goto done; }
+                    SVDC_TRACE_ADD(0, p0);
                     const uint32_t dst = a_base0 + ab * p.a_bytes;
                     mbar_arrive_expect_tx(bar.a_full + 8 * ab, p.a_bytes);
                     for (int kb = 0; kb < p.nkb; ++kb) {
@@ -248,7 +252,9 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
                 ++ui;
                 for (int cg = un.c0; cg < un.c1; cg += p.gc, ++ig) {
                     const uint32_t vs = ig % p.v_slots;
+                    SVDC_TRACE_MARK(p1);
                     if (!mbar_wait(bar.v_empty + 8 * vs, ((ig / p.v_slots) & 1u) ^ 1u, abort_flag, 2)) { record_timeout(p, abort_flag); goto done; }
+                    SVDC_TRACE_ADD(1, p1);
                     const uint32_t vdst = v_base0 + vs * p.vslice_bytes;
                     mbar_arrive_expect_tx(bar.v_full + 8 * vs, p.vslice_bytes);
                     for (int kb = 0; kb < p.nkb; ++kb)
@@ -257,7 +263,9 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
                     const int ce = min(cg + p.gc, un.c1);
                     for (int c = cg; c < ce; ++c, ++it) {
                         const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
+                        SVDC_TRACE_MARK(p2);
                         if (!mbar_wait(bar.empty + 8 * s, ph ^ 1u, abort_flag, 3)) { record_timeout(p, abort_flag); goto done; }
+                        SVDC_TRACE_ADD(2, p2);
                         mbar_arrive_expect_tx(bar.full + 8 * s, kTileBytes);
                         tma_load_3d(stage0 + s * kTileBytes, &tm_r, bar.full + 8 * s, c * kTileCols, un.rt * kTileRows, un.b);
                     }
@@ -273,30 +281,56 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
                 const Unit un = decode_unit(p, u);
                 if (*(volatile uint32_t *)&header_of(p, un.b)->full_steps == 0) continue;
                 const uint32_t ab = ui % p.a_bufs;
+                SVDC_TRACE_MARK(m0);
                 if (!mbar_wait(bar.a_full + 8 * ab, (ui / p.a_bufs) & 1u, abort_flag, 4)) { record_timeout(p, abort_flag); goto done; }
+                SVDC_TRACE_ADD(0, m0);
                 const uint64_t a_desc0 = smem_desc_kmajor(a_base0 + ab * p.a_bytes, p.kb_bytes);
                 for (int cg = un.c0; cg < un.c1; cg += p.gc, ++ig) {
                     const uint32_t vs = ig % p.v_slots, as = ig % p.acc_stages;
                     const int nsub = min(p.gc, un.c1 - cg);
+                    SVDC_TRACE_MARK(m1);
                     if (!mbar_wait(bar.v_full + 8 * vs, (ig / p.v_slots) & 1u, abort_flag, 5)) { record_timeout(p, abort_flag); goto done; }
+                    SVDC_TRACE_ADD(1, m1);
+                    SVDC_TRACE_MARK(m2);
                     if (!mbar_wait(bar.acc_empty + 8 * as, ((ig / p.acc_stages) & 1u) ^ 1u, abort_flag, 6)) { record_timeout(p, abort_flag); goto done; }
+                    SVDC_TRACE_ADD(2, m2);
                     tc_fence_after();
+                    SVDC_TRACE_MARK(m3);
                     const uint32_t idesc = idesc_bf16(kTileRows, nsub * kTileCols);
-                    const uint32_t d_tmem = tmem_base + as * p.acc_cols;
+                    const uint32_t d_tmem = tmem_base + as * p.acc_stride;
                     const uint64_t v_desc0 = smem_desc_kmajor(v_base0 + vs * p.vslice_bytes, p.kb_bytes);
-                    uint32_t acc = 0;
-                    for (int part = 0; part < 2; ++part)
+                    if (p.dual) {
+                        // Narrow groups (N <= 128) leave a dependent MMA chain latency-bound: the hi and the
+                        // lo part of the operand go to accumulators of their own, issued alternately, and
+                        // the epilogue adds the two.
+                        const uint32_t d_lo = d_tmem + p.acc_cols;
+                        uint32_t acc = 0;
                         for (int kb = 0; kb < p.nkb; ++kb) {
-                            // descriptors address in 16-byte units: add byte offsets >> 4
-                            const uint64_t a_kb = a_desc0 + ((part * p.a_half_bytes + kb * (kTileRows * p.kb_bytes)) >> 4);
+                            const uint64_t a_hi = a_desc0 + ((kb * (kTileRows * p.kb_bytes)) >> 4);
+                            const uint64_t a_lo = a_hi + (p.a_half_bytes >> 4);
                             const uint64_t v_kb = v_desc0 + ((kb * (p.gc * kTileCols * p.kb_bytes)) >> 4);
                             for (int ks = 0; ks < ksteps; ++ks) {
-                                mma_bf16_ss(d_tmem, a_kb + 2 * ks, v_kb + 2 * ks, idesc, acc);
+                                mma_bf16_ss(d_tmem, a_hi + 2 * ks, v_kb + 2 * ks, idesc, acc);
+                                mma_bf16_ss(d_lo, a_lo + 2 * ks, v_kb + 2 * ks, idesc, acc);
                                 acc = 1;
                             }
                         }
+                    } else {
+                        uint32_t acc = 0;
+                        for (int part = 0; part < 2; ++part)
+                            for (int kb = 0; kb < p.nkb; ++kb) {
+                                // descriptors address in 16-byte units: add byte offsets >> 4
+                                const uint64_t a_kb = a_desc0 + ((part * p.a_half_bytes + kb * (kTileRows * p.kb_bytes)) >> 4);
+                                const uint64_t v_kb = v_desc0 + ((kb * (p.gc * kTileCols * p.kb_bytes)) >> 4);
+                                for (int ks = 0; ks < ksteps; ++ks) {
+                                    mma_bf16_ss(d_tmem, a_kb + 2 * ks, v_kb + 2 * ks, idesc, acc);
+                                    acc = 1;
+                                }
+                            }
+                    }
                     mma_commit(bar.v_empty + 8 * vs);
                     mma_commit(bar.acc_full + 8 * as);
+                    SVDC_TRACE_ADD(3, m3);
                 }
                 mma_commit(bar.a_empty + 8 * ab);
                 ++ui;
@@ -316,22 +350,38 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
                 const uint32_t as = ig % p.acc_stages, aph = (ig / p.acc_stages) & 1u;
                 const int nsub = min(p.gc, un.c1 - cg);
                 const int last_own = last_own_chunk(it, nsub, grp);
+                SVDC_TRACE_MARK(e0);
                 if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar.acc_full + 8 * as, aph, abort_flag, 7))) { record_timeout(p, abort_flag); goto done; }
+                SVDC_TRACE_ADD(0, e0);
                 if (last_own < 0 && lane == 0) mbar_arrive(bar.acc_empty + 8 * as);
                 for (int j = 0; j < nsub; ++j, ++it) {
                     if ((it & 1u) != grp) continue;
                     const int c = cg + j;
                     const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
+                    SVDC_TRACE_MARK(e1);
                     if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar.full + 8 * s, ph, abort_flag, 8))) { record_timeout(p, abort_flag); goto done; }
+                    SVDC_TRACE_ADD(1, e1);
+                    SVDC_TRACE_MARK(e2);
                     tc_fence_after();
                     const uint32_t tile = stage0 + s * kTileBytes + (uint32_t)row * 128u;
-                    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + as * p.acc_cols + j * kTileCols;
+                    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + as * p.acc_stride + j * kTileCols;
                     uint32_t acc0[32], acc1[32];
                     tmem_ld_32x32(taddr, acc0);
                     tmem_ld_32x32(taddr + 32, acc1);
                     uint4 t[8];
 #pragma unroll
                     for (int cc = 0; cc < 8; ++cc) t[cc] = lds128(tile + (((uint32_t)cc) ^ ((uint32_t)row & 7u)) * 16u);
+                    if (p.dual) {   // product = hi-part accumulator + lo-part accumulator
+                        uint32_t lo0[32], lo1[32];
+                        tmem_ld_32x32(taddr + p.acc_cols, lo0);
+                        tmem_ld_32x32(taddr + p.acc_cols + 32, lo1);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            acc0[i] = __float_as_uint(__uint_as_float(acc0[i]) + __uint_as_float(lo0[i]));
+                            acc1[i] = __float_as_uint(__uint_as_float(acc1[i]) + __uint_as_float(lo1[i]));
+                        }
+                    }
                     tmem_wait_ld();
                     tc_fence_before();
                     __syncwarp();
@@ -351,6 +401,8 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
                         mbar_arrive(bar.empty + 8 * s);
                     }
                     __syncwarp();
+                    SVDC_TRACE_ADD(2, e2);
+                    SVDC_TRACE_COUNT(3);
                 }
             }
         }
@@ -358,6 +410,7 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
     }
 
 done:
+    SVDC_TRACE_FLUSH(g_trace);
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -1016,6 +1069,9 @@ size_t smem_bytes_full(const UmmaParams &p) {
 bool fill_cached(const StepArgs &a, UmmaParams &p) {
     if (!fill_params(a, p)) return false;
     fill_groups(a, p);
+    p.dual = p.gc <= 2 ? 1 : 0;
+    p.acc_stride = p.acc_cols * (p.dual ? 2 : 1);
+    p.acc_stages = 512 / p.acc_stride < kAccStages ? 512 / p.acc_stride : kAccStages;
     const size_t avail = kSmemBudget - 1024 /*alignment*/ - kBarBytes - 64;
     const size_t fixed = (size_t)p.v_slots * p.vslice_bytes;
     p.a_bufs = (2 * (size_t)p.a_bytes + fixed + 6 * (size_t)kTileBytes <= avail) ? 2 : 1;
