@@ -40,7 +40,7 @@ NOMINAL_HBM_GBS = 8000.0
 # profiles/umma_cached_kernel_flux_8blocks.txt: taken on 8 blocks of the same shape and
 # scaled by the block count (traffic is proportional to the blocks a launch covers).  The
 # tail of the output that is still in L2 when the kernel ends is not in the counter.
-NCU_TRAFFIC_BYTES_PER_BLOCK = {("flux", 2): 51907520}
+NCU_TRAFFIC_BYTES_PER_BLOCK = {("flux", 2): 51971616}
 
 
 def algorithmic_bytes(spec: streams.StreamSpec, nblocks: int):
@@ -156,8 +156,16 @@ def build_workload(spec, nblocks, device, block_offset=0, calibrate_rows=None):
         blk = block_offset + b
         st = streams.BlockStream(spec, blk, trajectory=0, device=device)
         st.features(0, out=F[b])
-        cal = streams.BlockStream(spec, blk, trajectory=1, device=device, rows=n_cal)
-        stack = cal.features(0)
+        if n_cal <= N:
+            cal = streams.BlockStream(spec, blk, trajectory=1, device=device, rows=n_cal)
+            stack = cal.features(0)
+        else:   # several snapshots of the calibration trajectories, as many rows as asked for
+            snaps = (n_cal + N - 1) // N
+            per_traj = len(spec.calib_timesteps)
+            stack = streams.calibration_stack(spec, blk, device=device,
+                                              trajectories=tuple(range(1, 1 + (snaps + per_traj - 1) // per_traj)),
+                                              timesteps=spec.calib_timesteps[:min(per_traj, snaps)])[:n_cal]
+            cal = None
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         Vk, lam, tr, info = sc.svdcache_calibrate(stack, k, workspace=ws, strict=False)
@@ -186,7 +194,8 @@ def run_ours(args):
 
     spec = streams.SPECS[args.workload]
     nblocks = args.blocks or (spec.blocks if spec.name != "hunyuan" else 8)
-    wl = build_workload(spec, nblocks, device, block_offset=rank_blocks(spec, rank, nblocks)[0])
+    wl = build_workload(spec, nblocks, device, block_offset=rank_blocks(spec, rank, nblocks)[0],
+                        calibrate_rows=args.calib_rows or None)
     F, bases, state, Fhat, dt = wl["F"], wl["bases"], wl["state"], wl["Fhat"], wl["dt"]
     k, beta, interval = spec.k, spec.beta, spec.interval
     bytes_full, bytes_cached = algorithmic_bytes(spec, nblocks)
@@ -478,6 +487,7 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--ref-rows", type=int, default=1024)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--calib-rows", type=int, default=0, help="rows of the per-block calibration stack (default: min(N, 4608))")
     ap.add_argument("--sweep", action="store_true", help="rank and calibration sweep on the FLUX shape")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
