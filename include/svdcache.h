@@ -167,11 +167,13 @@ SVDCACHE_API int svdcache_basis_prepare(const float *Vk, int D, int k, int dtype
 
 /* ---------------------------------------------------------------------------------
  * Per-block cache state, a caller-owned flat device buffer (checkpoint = memcpy):
- *   header (256 B) | Chat fp32 [N x k] | Chat operand copy | R dtype [N x D]   (dense, no pitch)
+ *   header (256 B) | Chat fp32 [N x k] | Chat operand copy | step scratch | R dtype [N x D]   (dense, no pitch)
  * The operand copy exists only for dtype = SVDCACHE_BF16: Chat as two bf16 arrays [N x k],
  * hi = bf16(Chat) and lo = bf16(Chat - hi), which every full step rewrites together with
  * Chat and the cached step feeds to the tensor cores as they are (hi + lo carries ~16
- * mantissa bits).  Offsets of Chat and R come from svdcache_state_layout.
+ * mantissa bits).  The step scratch (bf16 mode only) belongs to the full step: this step's
+ * coefficients C in the same split form, and four words per 128-row tile.  Offsets of Chat
+ * and R come from svdcache_state_layout.
  * The header counts the full steps the state has seen and carries a sticky device
  * status word.  svdcache_state_reset must be called once before first use (and again to
  * start a new sampling run): it clears the counter, so the next full step initialises
@@ -235,8 +237,11 @@ SVDCACHE_API int svdcache_cached_step_batched(int nblocks, const void *state, si
  *                      128-row tile between the two CTAs of a thread-block cluster
  *                      (each streams half of the columns; the partial coefficients
  *                      meet through distributed shared memory) where the shape
- *                      allows it.  Returns the previous setting.
- *   svdcache_last_path: which kernel family the last step call used (1, 2 or 3).
+ *                      allows it, 4 = as 2, with the experimental batched two-phase full
+ *                      step (every tile's columns shared by up to eight CTAs, partial
+ *                      coefficients combined through memory, pass 2 one or two batches
+ *                      after pass 1).  Returns the previous setting.
+ *   svdcache_last_path: which kernel family the last step call used (1 .. 4).
  * ------------------------------------------------------------------------------- */
 SVDCACHE_API uint64_t svdcache_kernel_launches(void);
 SVDCACHE_API int svdcache_set_path(int path);

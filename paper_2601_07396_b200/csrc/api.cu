@@ -43,13 +43,14 @@ static int dispatch(const StepArgs &a_in, bool full, cudaStream_t s) {
     const bool can_umma = umma_supported(a, full);
     if (want >= 2 && !can_umma) return SVDCACHE_ERR_BAD_SHAPE;
     const bool use_umma = (want >= 2) || (want == 0 && can_umma);
-    a.cluster_split = (want == 3) ? 1 : 0;
-    g_last_path.store(use_umma ? (want == 3 ? 3 : 2) : 1);
+    a.cluster_split = (want == 3) ? 1 : (want == 4) ? 2 : 0;
+    g_last_path.store(use_umma ? (want >= 3 ? want : 2) : 1);
     if (use_umma) return full ? umma_full_step(a, s) : umma_cached_step(a, s);
     return full ? simt_full_step(a, s) : simt_cached_step(a, s);
 }
 
-__global__ void state_reset_kernel(StateHeader *h, int64_t N, int D, int k, int dtype) {
+__global__ void state_reset_kernel(StateHeader *h, int64_t N, int D, int k, int dtype, uint32_t *sync, int sync_words) {
+    for (int i = threadIdx.x; i < sync_words; i += blockDim.x) sync[i] = 0u;   // per-tile counters and ready marks
     if (threadIdx.x == 0 && blockIdx.x == 0) {
         h->magic = kStateMagic;
         h->dtype = dtype;
@@ -89,7 +90,7 @@ const char *svdcache_last_cuda_error(void) { return g_cuda_error; }
 
 uint64_t svdcache_kernel_launches(void) { return g_launches.load(); }
 int svdcache_set_path(int path) {
-    if (path < 0 || path > 3) return SVDCACHE_ERR_INVALID_ARG;
+    if (path < 0 || path > 4) return SVDCACHE_ERR_INVALID_ARG;
     return g_path.exchange(path);
 }
 int svdcache_last_path(void) { return g_last_path.load(); }
@@ -220,7 +221,10 @@ int svdcache_state_reset(void *state, int64_t N, int D, int k, int dtype, void *
     if (rc) return rc;
     if (!state) return SVDCACHE_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(state) & 255u) != 0) return SVDCACHE_ERR_BAD_ALIGN;
-    state_reset_kernel<<<1, 32, 0, (cudaStream_t)stream>>>((StateHeader *)state, N, D, k, dtype);
+    const StateLayout SL = state_layout(N, D, k, dtype);
+    state_reset_kernel<<<1, 256, 0, (cudaStream_t)stream>>>((StateHeader *)state, N, D, k, dtype,
+                                                            reinterpret_cast<uint32_t *>((char *)state + SL.sync),
+                                                            (int)((SL.r - SL.sync) / 4));
     count_launch();
     return check_last_launch();
 }

@@ -49,18 +49,26 @@ inline BasisLayout basis_layout(int D, int k, int dtype) {
 }
 
 // header | Chat fp32 [N x k] | (bf16 only) Chat as a split-bf16 pair: hi [N x k], lo [N x k] |
-// R [N x D].  hi = bf16(Chat), lo = bf16(Chat - hi): the tensor-core operand of the cached
-// step, written by the full step next to Chat so that the cached step reads it as it is.
+// (bf16 only) scratch of the full step: this step's C as a split-bf16 pair, and four words per
+// 128-row tile (two arrival counters, ready mark) | R [N x D].
+// hi = bf16(x), lo = bf16(x - hi).  The pair of Chat is the tensor-core operand of the cached
+// step, written by the full step next to Chat so that the cached step reads it as it is; the
+// pair of C is the operand of the full step's own second pass.
 struct StateLayout {
-    size_t chat, op_hi, op_lo, r, total;
+    size_t chat, op_hi, op_lo, c_hi, c_lo, sync, r, total;
 };
 inline StateLayout state_layout(int64_t N, int D, int k, int dtype) {
     StateLayout L;
-    const size_t op = dtype == SVDCACHE_BF16 ? align_up((size_t)N * k * 2, kAlign) : 0;
+    const bool bf = dtype == SVDCACHE_BF16;
+    const size_t op = bf ? align_up((size_t)N * k * 2, kAlign) : 0;
+    const size_t tiles = (size_t)((N + 127) / 128);
     L.chat = kHeaderBytes;
     L.op_hi = L.chat + align_up((size_t)N * k * 4, kAlign);
     L.op_lo = L.op_hi + op;
-    L.r = L.op_lo + op;
+    L.c_hi = L.op_lo + op;
+    L.c_lo = L.c_hi + op;
+    L.sync = L.c_lo + op;
+    L.r = L.sync + (bf ? align_up(tiles * 16, kAlign) : 0);
     L.total = L.r + align_up((size_t)N * D * elem_bytes(dtype), kAlign);
     return L;
 }
@@ -84,7 +92,8 @@ struct StepArgs {
     int64_t N;
     int D, k, dtype, nblocks;
     float beta;
-    int cluster_split;      // full step, tcgen05 family: share each row tile between the two CTAs of a cluster
+    int cluster_split;      // full step, tcgen05 family: 1 = share each row tile between the two CTAs of a cluster,
+                            // 2 = batched two-phase schedule (column slices over CTAs, partials through memory)
 };
 
 // launch bookkeeping (api.cu)

@@ -132,6 +132,17 @@ def test_cluster_split_full_step(N, D, k):
     assert sc.svdcache_last_path() in (0, 2, 3)
 
 
+@pytest.mark.parametrize("N,D,k,ld_pad", [(300, 1152, 64, 0), (257, 3072, 128, 0), (1000, 512, 64, 0), (129, 3072, 64, 8),
+                                          (1, 64, 64, 0), (515, 1024, 16, 0), (384, 2048, 32, 64), (5000, 3072, 64, 0)])
+def test_two_phase_full_step(N, D, k, ld_pad):
+    """Path 4: the full step with every tile's columns shared by up to four CTAs, partial
+    coefficients combined through memory, pass 2 one batch later -- same oracle, same bounds.
+    (1, 64, 64) lies outside that schedule and must fall back silently."""
+    spec = streams.StreamSpec("twophase", blocks=1, rows=N, D=D, dtype="bf16", k=k, T=5, interval=2,
+                              rank=min(D, 2 * k), amp=30.0, power=1.0, noise_std=0.02)
+    _play(spec, 0, None, range(5), path=4, ld_pad=ld_pad)
+
+
 def test_batched_equals_per_block_and_oracle():
     spec = streams.StreamSpec("batch", blocks=3, rows=200, D=512, dtype="bf16", k=64, T=4, interval=2,
                               rank=128, amp=30.0, power=1.0, noise_std=0.02)
