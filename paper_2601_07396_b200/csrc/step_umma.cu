@@ -143,10 +143,6 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
     asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
                  : "memory");
 }
-__device__ __forceinline__ void sts64(uint32_t addr, uint32_t x, uint32_t y) {
-    asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(addr), "r"(x), "r"(y) : "memory");
-}
-
 // Every epilogue warp waits for every accumulator of the ring, in order, and arrives on its
 // "empty" barrier once per group -- after reading its last chunk of the group, or at once if
 // the group holds none of its chunks.  A waiter that skipped a phase of an mbarrier could
@@ -445,11 +441,6 @@ done:
 // ======================================================================================
 constexpr int kThreadsFull = 320;
 constexpr uint32_t kBlk32Bytes = kTileRows * 128u;   // 16 KB: 128 rows x 32 fp32 (or x 64 bf16)
-
-// 32 consecutive coefficients of one row: EMA against `prev`, global stores, split-bf16 pack.
-struct RowOut {
-    float *chat, *cout;          // global rows (nullptr: do not store)
-};
 
 __device__ __forceinline__ void load_row32(uint32_t row_addr, uint32_t row, uint32_t row_bytes, int ncols, float (&v)[32]) {
 #pragma unroll
