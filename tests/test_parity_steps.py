@@ -143,8 +143,20 @@ def test_two_phase_full_step(N, D, k, ld_pad):
     _play(spec, 0, None, range(5), path=4, ld_pad=ld_pad)
 
 
-def test_batched_equals_per_block_and_oracle():
-    spec = streams.StreamSpec("batch", blocks=3, rows=200, D=512, dtype="bf16", k=64, T=4, interval=2,
+@pytest.mark.parametrize("path,rows,D", [(0, 200, 512), (3, 200, 512), (4, 200, 512), (4, 700, 3072)])
+def test_batched_equals_per_block_and_oracle(path, rows, D):
+    """One batched launch over three blocks against three per-block launches (bitwise) and the
+    oracle; for the default kernels and for the two opt-in schedules of the full step (whose
+    tiles run across block boundaries)."""
+    prev = sc.svdcache_set_path(path)
+    try:
+        _batched_case(rows, D)
+    finally:
+        sc.svdcache_set_path(prev)
+
+
+def _batched_case(rows, D):
+    spec = streams.StreamSpec("batch", blocks=3, rows=rows, D=D, dtype="bf16", k=64, T=4, interval=2,
                               rank=128, amp=30.0, power=1.0, noise_std=0.02)
     nb, N, D, k, dt = 3, spec.rows, spec.D, spec.k, sc.BF16
     bases = torch.stack([sc.svdcache_basis_prepare(
