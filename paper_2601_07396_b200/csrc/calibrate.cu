@@ -21,7 +21,9 @@ namespace svdc {
 
 // tensor-core Gram (gram_umma.cu)
 bool umma_gram_supported(int64_t M, int D, int64_t ld, int dtype);
-int umma_gram_accumulate(const void *F, int64_t M, int D, int64_t ld, double *G, int *status, cudaStream_t s);
+int umma_gram_accumulate(const void *F, int64_t M, int D, int64_t ld, double *G, double *scratch, int *status,
+                         cudaStream_t s);
+size_t umma_gram_scratch_bytes(int D);
 
 namespace {
 
@@ -38,7 +40,7 @@ int ritz_width(int D, int k) {
 }
 
 struct CalibLayout {
-    size_t G, Q, Z, T, S, W, X, theta, resid, scal, dead, total;
+    size_t G, gram_scratch, Q, Z, T, S, W, X, theta, resid, scal, dead, total;
     int m;
 };
 
@@ -48,6 +50,7 @@ CalibLayout calib_layout(int D, int k) {
     const size_t dm = align_up((size_t)D * L.m * 8, kAlign), mm = align_up((size_t)L.m * L.m * 8, kAlign);
     size_t at = kHeaderBytes;
     L.G = at; at += align_up((size_t)D * D * 8, kAlign);
+    L.gram_scratch = at; at += align_up(umma_gram_scratch_bytes(D), kAlign);   // depends on D only, like G
     L.Q = at; at += dm;
     L.Z = at; at += dm;
     L.T = at; at += dm;
@@ -464,7 +467,9 @@ int calib_accumulate(const void *F, int64_t M, int D, int64_t ld, int dtype, voi
     double *G = (double *)(w + kHeaderBytes);
     int rc;
     if (umma_gram_supported(M, D, ld, dtype)) {
-        rc = umma_gram_accumulate(F, M, D, ld, G, &reinterpret_cast<CalibHeader *>(w)->status, s);
+        const CalibLayout L = calib_layout(D, 8);
+        double *scratch = umma_gram_scratch_bytes(D) ? (double *)(w + L.gram_scratch) : nullptr;
+        rc = umma_gram_accumulate(F, M, D, ld, G, scratch, &reinterpret_cast<CalibHeader *>(w)->status, s);
     } else if (dtype == SVDCACHE_BF16) {
         const __nv_bfloat16 *f = (const __nv_bfloat16 *)F;
         rc = dgemm<__nv_bfloat16, __nv_bfloat16, true>(f, ld, f, ld, G, D, D, D, M, true, true, s);

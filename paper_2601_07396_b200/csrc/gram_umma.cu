@@ -12,7 +12,11 @@
 // overlaps the MMAs of the next.
 //
 // One CTA owns one 128 x 256 tile of G's upper block triangle for the whole call, and walks
-// its chunks in order: no atomics, a fixed summation order, bit-reproducible results.
+// its chunks in order: no atomics, a fixed summation order, bit-reproducible results.  When
+// there are a few more tiles than SMs (D = 3072: 156 tiles, 148 SMs), the surplus tiles are
+// not left to a nearly empty second wave: each is cut along the stack rows into segments,
+// one per CTA, that sum into private fp64 partial tiles, and a small kernel adds those to G
+// in segment order afterwards.
 // Warp roles (192 threads): 0 = TMA producer, 1 = MMA issuer (+ TMEM owner), 2..5 = flush.
 #include "internal.cuh"
 #include "umma.cuh"
@@ -39,6 +43,10 @@ struct GramParams {
     int D;
     int tiles_j;          // 256-column tiles per row of tiles
     int ntiles;
+    int whole;            // tiles [0, whole) are summed over the whole stack by one CTA each, into G
+    int nseg;             // each tile of [whole, ntiles) is cut into nseg row segments (units after the whole tiles)
+    int units;            // whole + (ntiles - whole) * nseg
+    double *partials;     // one dense 128 x 256 fp64 tile per segment unit
     double *G;
     int *status;          // device word that receives SVDCACHE_ERR_TIMEOUT if a bounded wait runs out
 };
@@ -53,6 +61,26 @@ __device__ __forceinline__ void decode_tile(const GramParams &p, int t, int &ti,
         if (t < n) { tj = first + t; return; }
         t -= n;
     }
+}
+
+struct GramUnit {
+    int tile, st_lo, st_hi;   // tile, stage range [st_lo, st_hi) of the stack
+    double *out;              // partial tile, or nullptr: the tile of G itself
+    int store_first;          // 1: the first chunk overwrites (partial tiles start undefined)
+};
+__device__ __forceinline__ GramUnit decode_gram_unit(const GramParams &p, int u, int nstages_total) {
+    GramUnit x;
+    if (u < p.whole) {
+        x.tile = u; x.st_lo = 0; x.st_hi = nstages_total; x.out = nullptr; x.store_first = 0;
+    } else {
+        const int idx = u - p.whole, seg = idx % p.nseg;
+        x.tile = p.whole + idx / p.nseg;
+        x.st_lo = (int)(((int64_t)seg * nstages_total) / p.nseg);
+        x.st_hi = (int)(((int64_t)(seg + 1) * nstages_total) / p.nseg);
+        x.out = p.partials + (size_t)idx * (kGTileI * kGTileJ);
+        x.store_first = 1;
+    }
+    return x;
 }
 
 // MN-major operand descriptor, 128-byte swizzle: 64-element blocks along M/N are `lbo` bytes
@@ -99,12 +127,13 @@ umma_gram_kernel(const __grid_constant__ CUtensorMap tm_f, const GramParams p) {
     if (warp == 0) {
         if (lane == 0) {
             uint32_t it = 0;
-            for (int t = blockIdx.x; t < p.ntiles; t += gridDim.x) {
+            for (int u = blockIdx.x; u < p.units; u += gridDim.x) {
+                const GramUnit gu = decode_gram_unit(p, u, nstages_total);
                 int ti, tj;
-                decode_tile(p, t, ti, tj);
+                decode_tile(p, gu.tile, ti, tj);
                 const int i0 = ti * kGTileI, j0 = tj * kGTileJ;
                 const int nj = min(kGTileJ, p.D - j0) / kGBlk;
-                for (int st = 0; st < nstages_total; ++st, ++it) {
+                for (int st = gu.st_lo; st < gu.st_hi; ++st, ++it) {
                     const uint32_t s = it % kGStages, ph = (it / kGStages) & 1u;
                     if (!mbar_wait(empty + 8 * s, ph ^ 1u, abort_flag, 1)) goto done;
                     const uint32_t dst = base + s * kGStageBytes;
@@ -119,16 +148,17 @@ umma_gram_kernel(const __grid_constant__ CUtensorMap tm_f, const GramParams p) {
     } else if (warp == 1) {
         if (lane == 0) {
             uint32_t it = 0, ic = 0;
-            for (int t = blockIdx.x; t < p.ntiles; t += gridDim.x) {
+            for (int u = blockIdx.x; u < p.units; u += gridDim.x) {
+                const GramUnit gu = decode_gram_unit(p, u, nstages_total);
                 int ti, tj;
-                decode_tile(p, t, ti, tj);
+                decode_tile(p, gu.tile, ti, tj);
                 const int nj = min(kGTileJ, p.D - tj * kGTileJ) / kGBlk;
                 const uint32_t idesc = idesc_bf16_mnmajor(kGTileI, nj * kGBlk);
-                for (int st0 = 0; st0 < nstages_total; st0 += kChunkStages, ++ic) {
+                for (int st0 = gu.st_lo; st0 < gu.st_hi; st0 += kChunkStages, ++ic) {
                     const uint32_t buf = ic & 1u;
                     if (!mbar_wait(acc_empty + 8 * buf, ((ic >> 1) & 1u) ^ 1u, abort_flag, 2)) goto done;
                     tc_fence_after();
-                    const int st1 = min(st0 + kChunkStages, nstages_total);
+                    const int st1 = min(st0 + kChunkStages, gu.st_hi);
                     for (int st = st0; st < st1; ++st, ++it) {
                         const uint32_t s = it % kGStages, ph = (it / kGStages) & 1u;
                         if (!mbar_wait(full + 8 * s, ph, abort_flag, 3)) goto done;
@@ -149,13 +179,15 @@ umma_gram_kernel(const __grid_constant__ CUtensorMap tm_f, const GramParams p) {
         // flush: G[i0 + row][j0 ...] += accumulator row (thread = TMEM lane = tile row)
         const int q = warp & 3, row = q * 32 + lane;
         uint32_t ic = 0;
-        for (int t = blockIdx.x; t < p.ntiles; t += gridDim.x) {
+        for (int u = blockIdx.x; u < p.units; u += gridDim.x) {
+            const GramUnit gu = decode_gram_unit(p, u, nstages_total);
             int ti, tj;
-            decode_tile(p, t, ti, tj);
+            decode_tile(p, gu.tile, ti, tj);
             const int i0 = ti * kGTileI, j0 = tj * kGTileJ;
             const int ncols = min(kGTileJ, p.D - j0);
-            double *grow = p.G + (size_t)(i0 + row) * p.D + j0;
-            for (int st0 = 0; st0 < nstages_total; st0 += kChunkStages, ++ic) {
+            double *grow = gu.out ? gu.out + (size_t)row * kGTileJ : p.G + (size_t)(i0 + row) * p.D + j0;
+            for (int st0 = gu.st_lo; st0 < gu.st_hi; st0 += kChunkStages, ++ic) {
+                const bool overwrite = gu.store_first && st0 == gu.st_lo;
                 const uint32_t buf = ic & 1u;
                 if (!__all_sync(0xFFFFFFFFu, mbar_wait(acc_full + 8 * buf, (ic >> 1) & 1u, abort_flag, 4))) goto done;
                 tc_fence_after();
@@ -165,7 +197,8 @@ umma_gram_kernel(const __grid_constant__ CUtensorMap tm_f, const GramParams p) {
                     tmem_ld_32x32(taddr + c0, acc);
                     double2 g[16];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) g[i] = *reinterpret_cast<const double2 *>(grow + c0 + 2 * i);
+                    for (int i = 0; i < 16; ++i)
+                        g[i] = overwrite ? make_double2(0.0, 0.0) : *reinterpret_cast<const double2 *>(grow + c0 + 2 * i);
                     tmem_wait_ld();
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
@@ -190,6 +223,26 @@ done:
     }
 }
 
+// G tile += its partial tiles, in segment order (one thread per element)
+__global__ void gram_reduce_kernel(GramParams p) {
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;           // element within a tile
+    const int x = blockIdx.y;                                      // which split tile
+    if (e >= kGTileI * kGTileJ) return;
+    int ti, tj;
+    decode_tile(p, p.whole + x, ti, tj);
+    const int r = e / kGTileJ, c = e % kGTileJ;
+    const int j = tj * kGTileJ + c;
+    if (j >= p.D) return;
+    const int nstages_total = (int)((p.M + kGStageRows - 1) / kGStageRows);
+    double acc = 0.0;
+    for (int s = 0; s < p.nseg; ++s) {
+        const GramUnit gu = decode_gram_unit(p, p.whole + x * p.nseg + s, nstages_total);
+        if (gu.st_hi > gu.st_lo)   // a short stack leaves some segments empty: their partial tiles were never written
+            acc += p.partials[((size_t)x * p.nseg + s) * (kGTileI * kGTileJ) + e];
+    }
+    p.G[(size_t)(ti * kGTileI + r) * p.D + j] += acc;
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
@@ -206,6 +259,8 @@ EncodeTiledFn gram_encode_fn() {
     }();
     return fn;
 }
+
+constexpr int kNominalSMs = 148;   // the split of surplus tiles is sized for this many CTAs
 
 int gram_tiles(int D, int *tiles_j) {
     const int ti_n = D / kGTileI, tj_n = (D + kGTileJ - 1) / kGTileJ;
@@ -227,7 +282,24 @@ bool umma_gram_supported(int64_t M, int D, int64_t ld, int dtype) {
     return gram_encode_fn() != nullptr;
 }
 
-int umma_gram_accumulate(const void *F, int64_t M, int D, int64_t ld, double *G, int *status, cudaStream_t s) {
+// surplus tiles (beyond one per SM) and the segments each is cut into; 0 / 1 when the split does not apply
+static void gram_split(int ntiles, int *surplus, int *nseg) {
+    *surplus = 0; *nseg = 1;
+    const int e = ntiles - kNominalSMs;
+    if (e > 0 && e <= kNominalSMs / 2) { *surplus = e; *nseg = kNominalSMs / e; }
+}
+
+// bytes of the partial tiles (depends on D only)
+size_t umma_gram_scratch_bytes(int D) {
+    if (D < 256 || (D % kGTileI) != 0) return 0;
+    int tj, surplus, nseg;
+    const int ntiles = gram_tiles(D, &tj);
+    gram_split(ntiles, &surplus, &nseg);
+    return (size_t)surplus * nseg * kGTileI * kGTileJ * sizeof(double);
+}
+
+int umma_gram_accumulate(const void *F, int64_t M, int D, int64_t ld, double *G, double *scratch, int *status,
+                         cudaStream_t s) {
     EncodeTiledFn fn = gram_encode_fn();
     if (!fn) return SVDCACHE_ERR_CUDA;
     CUtensorMap tm;
@@ -242,6 +314,16 @@ int umma_gram_accumulate(const void *F, int64_t M, int D, int64_t ld, double *G,
     GramParams p{};
     p.M = M; p.D = D; p.G = G; p.status = status;
     p.ntiles = gram_tiles(D, &p.tiles_j);
+    int sms = 0, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (sms <= 0) sms = kNominalSMs;
+    int surplus = 0, nseg = 1;
+    if (sms == kNominalSMs && scratch) gram_split(p.ntiles, &surplus, &nseg);
+    p.whole = p.ntiles - surplus;
+    p.nseg = nseg;
+    p.units = p.whole + surplus * nseg;
+    p.partials = scratch;
     const size_t smem = 1024 + (size_t)kGStages * kGStageBytes + kGBarBytes + 64;
     static bool attr_set = false;
     if (!attr_set) {
@@ -249,13 +331,13 @@ int umma_gram_accumulate(const void *F, int64_t M, int D, int64_t ld, double *G,
         if (rc) return rc;
         attr_set = true;
     }
-    int sms = 0, dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (sms <= 0) sms = 148;
-    const int grid = p.ntiles < sms ? p.ntiles : sms;
+    const int grid = p.units < sms ? p.units : sms;
     umma_gram_kernel<<<grid, kGThreads, smem, s>>>(tm, p);
     count_launch();
+    if (surplus > 0) {
+        gram_reduce_kernel<<<dim3((kGTileI * kGTileJ + 255) / 256, surplus), 256, 0, s>>>(p);
+        count_launch();
+    }
     return check_last_launch();
 }
 
