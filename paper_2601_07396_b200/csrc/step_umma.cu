@@ -435,11 +435,13 @@ done:
 // next unit runs while the epilogue still drains this one.  The producer requests each basis
 // slice one group ahead of the F chunks that go with it.
 //
-// Warp roles (320 threads): 0 = TMA producer, 1 = MMA issuer (+ TMEM owner), 2..5 = epilogue
-// group 0, 6..9 = C warps, which turn into epilogue group 1 once the A operand is written
-// (pass 2 cannot start before that, so the two jobs never overlap).
+// Warp roles (352 threads): 0 = TMA producer of the F chunks, 10 = TMA producer of the basis
+// slices, 1 = MMA issuer (+ TMEM owner), 2..5 = epilogue group 0, 6..9 = C warps, which turn
+// into epilogue group 1 once the A operand is written (pass 2 cannot start before that, so
+// the two jobs never overlap).
 // ======================================================================================
-constexpr int kThreadsFull = 320;
+constexpr int kThreadsFull = 352;
+constexpr int kFullVWarp = 10;   // second TMA producer (basis slices); warps 2..9 are the epilogue
 constexpr uint32_t kBlk32Bytes = kTileRows * 128u;   // 16 KB: 128 rows x 32 fp32 (or x 64 bf16)
 
 __device__ __forceinline__ void load_row32(uint32_t row_addr, uint32_t row, uint32_t row_bytes, int ncols, float (&v)[32]) {
@@ -538,68 +540,61 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer ---
+        // ---------------------------------------------------- TMA producer: F chunks ---
+        // Two request streams feed the tensor cores: F chunks (ring of p.stages slots) and basis
+        // slices (ring of p.v_slots slots), both in (unit, pass, group) order.  Neither may hold
+        // the other up -- a blocked F ring must not delay the next basis slice, and the other way
+        // round -- so each stream has a thread of its own (this one, and warp 10), each a plain
+        // loop of wait / expect / copy: a single thread polling both rings spent ~1200 cycles per
+        // chunk on its own serial instruction chain and was the bottleneck of the kernel.
         if (lane == 0) {
             const uint64_t pol_keep = policy_evict_last(), pol_drop = policy_evict_first();
-            // Two request streams share this thread: F chunks (ring of p.stages slots) and basis
-            // slices (ring of p.v_slots slots), both in (unit, pass, group) order.  Neither may
-            // hold the other up -- a blocked F ring must not delay the next basis slice, and the
-            // other way round -- so the thread polls both rings without blocking.
-            struct Step { int u, pass, g; };
-            auto next_step = [&](Step x) {
-                if (++x.g == G) { x.g = 0; if (++x.pass == 2) { x.pass = 0; x.u += nclusters; } }
-                return x;
-            };
-            Step vcur{cid, 0, 0}, fcur{cid, 0, 0};
-            uint32_t iv = 0, it = 0;   // basis slices, F chunks requested so far
-            int fc = 0;                // next chunk of fcur's group (offset within the group)
-            long long t_idle = clock64();
-            SVDC_TRACE_MARK(tp);
-            while (fcur.u < p.units || vcur.u < p.units) {
-                bool progress = false;
-                if (vcur.u < p.units) {
-                    const uint32_t vs = iv % p.v_slots;
-                    if (mbar_test_wait(bar.v_empty + 8 * vs, ((iv / p.v_slots) & 1u) ^ 1u)) {
-                        const Unit un = decode_unit(p, vcur.u);
-                        const int cg = (g_off + (vcur.pass == 0 ? vcur.g : G - 1 - vcur.g)) * p.gc;
+            uint32_t it = 0, s = 0, ph = 0;   // F chunks requested so far; ring slot and phase of the next one
+            for (int u = cid; u < p.units; u += nclusters) {
+                const Unit un = decode_unit(p, u);
+                for (int pass = 0; pass < 2; ++pass)
+                    for (int g = 0; g < G; ++g) {
+                        const int cg = (g_off + (pass == 0 ? g : G - 1 - g)) * p.gc;
+                        const int nsub = min(p.gc, CT - cg);
+                        for (int j = 0; j < nsub; ++j, ++it) {
+                            if (!mbar_wait(bar.empty + 8 * s, ph ^ 1u, abort_flag, 100)) {
+                                record_timeout(p, abort_flag, it, (uint32_t)(pass * 100 + g));
+                                goto done;
+                            }
+                            mbar_arrive_expect_tx(bar.full + 8 * s, kTileBytes);
+                            tma_load_3d_hint(stage0 + s * kTileBytes, &tm_f, bar.full + 8 * s, (cg + j) * kTileCols,
+                                             un.rt * kTileRows, un.b, pass == 0 ? pol_keep : pol_drop);
+                            if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; }
+                        }
+                    }
+            }
+        }
+    } else if (warp == kFullVWarp) {
+        // ------------------------------------------------ TMA producer: basis slices ---
+        if (lane == 0) {
+            uint32_t iv = 0, vs = 0, vph = 0;
+            for (int u = cid; u < p.units; u += nclusters) {
+                const Unit un = decode_unit(p, u);
+                for (int pass = 0; pass < 2; ++pass)
+                    for (int g = 0; g < G; ++g, ++iv) {
+                        const int cg = (g_off + (pass == 0 ? g : G - 1 - g)) * p.gc;
+                        if (!mbar_wait(bar.v_empty + 8 * vs, vph ^ 1u, abort_flag, 101)) {
+                            record_timeout(p, abort_flag, iv, (uint32_t)(pass * 100 + g));
+                            goto done;
+                        }
                         const uint32_t vdst = v_base0 + vs * p.vslice_bytes;
                         mbar_arrive_expect_tx(bar.v_full + 8 * vs, p.vslice_bytes);
-                        if (vcur.pass == 0) {   // V_k^T columns of each chunk: gc boxes of k rows x 64
+                        if (pass == 0) {   // V_k^T columns of each chunk: gc boxes of k rows x 64
                             for (int j = 0; j < p.gc; ++j)
                                 tma_load_3d(vdst + j * (p.k * 128), &tm_vt, bar.v_full + 8 * vs, (cg + j) * kTileCols, 0, un.b);
-                        } else {                // V_k rows of the group: one box of gc*64 rows per K block
+                        } else {           // V_k rows of the group: one box of gc*64 rows per K block
                             for (int kb = 0; kb < p.nkb; ++kb)
                                 tma_load_3d(vdst + kb * (p.gc * kTileCols * p.kb_bytes), &tm_v, bar.v_full + 8 * vs,
                                             kb * p.kb_elems, cg * kTileCols, un.b);
                         }
-                        vcur = next_step(vcur);
-                        ++iv;
-                        progress = true;
+                        if (++vs == (uint32_t)p.v_slots) { vs = 0; vph ^= 1u; }
                     }
-                }
-                if (fcur.u < p.units) {
-                    const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                    if (mbar_test_wait(bar.empty + 8 * s, ph ^ 1u)) {
-                        const Unit un = decode_unit(p, fcur.u);
-                        const int cg = (g_off + (fcur.pass == 0 ? fcur.g : G - 1 - fcur.g)) * p.gc;
-                        const int nsub = min(p.gc, CT - cg);
-                        mbar_arrive_expect_tx(bar.full + 8 * s, kTileBytes);
-                        tma_load_3d_hint(stage0 + s * kTileBytes, &tm_f, bar.full + 8 * s, (cg + fc) * kTileCols,
-                                         un.rt * kTileRows, un.b, fcur.pass == 0 ? pol_keep : pol_drop);
-                        ++it;
-                        if (++fc == nsub) { fc = 0; fcur = next_step(fcur); }
-                        progress = true;
-                    }
-                }
-                if (progress) {
-                    t_idle = clock64();
-                } else if (*abort_flag || clock64() - t_idle > kWaitCycles) {
-                    atomicCAS(const_cast<int *>(abort_flag), 0, 100);
-                    record_timeout(p, abort_flag, it, iv, (uint32_t)(fcur.pass * 100 + fcur.g) << 16 | (uint32_t)(vcur.pass * 100 + vcur.g));
-                    goto done;
-                }
             }
-            SVDC_TRACE_ADD(0, tp);
         }
     } else if (warp == 1) {
         // -------------------------------------------------------------- MMA issuer ---
