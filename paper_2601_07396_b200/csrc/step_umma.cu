@@ -143,6 +143,15 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
     asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
                  : "memory");
 }
+// Position in a ring of n slots -- slot index and phase parity -- advanced without dividing:
+// the roles below are serial instruction chains, and a division by a run-time ring size
+// costs each of them ~100 cycles per chunk.
+struct RingPos {
+    uint32_t idx = 0, ph = 0;
+    __device__ __forceinline__ void step(uint32_t n) { if (++idx == n) { idx = 0; ph ^= 1u; } }
+    __device__ __forceinline__ void skip(uint32_t k, uint32_t n) { const uint32_t t = idx + k; idx = t % n; ph ^= (t / n) & 1u; }
+};
+
 // Every epilogue warp waits for every accumulator of the ring, in order, and arrives on its
 // "empty" barrier once per group -- after reading its last chunk of the group, or at once if
 // the group holds none of its chunks.  A waiter that skipped a phase of an mbarrier could
@@ -222,7 +231,8 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer ---
         if (lane == 0) {
-            uint32_t it = 0, ig = 0, ui = 0, ua = 0;   // chunks, groups, units started; A tiles requested
+            uint32_t ui = 0, ua = 0;                   // units started; A tiles requested
+            RingPos fr, vr;                            // next R slot, next basis slot
             int u_a = blockIdx.x;                      // unit cursor of the A-tile requests (runs ahead)
             for (int u = blockIdx.x; u < p.units; u += gridDim.x) {
                 const Unit un = decode_unit(p, u);
@@ -250,10 +260,11 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
                     ++ua;
                 }
                 ++ui;
-                for (int cg = un.c0; cg < un.c1; cg += p.gc, ++ig) {
-                    const uint32_t vs = ig % p.v_slots;
+                for (int cg = un.c0; cg < un.c1; cg += p.gc) {
+                    const uint32_t vs = vr.idx;
                     SVDC_TRACE_MARK(p1);
-                    if (!mbar_wait(bar.v_empty + 8 * vs, ((ig / p.v_slots) & 1u) ^ 1u, abort_flag, 2)) { record_timeout(p, abort_flag); goto done; }
+                    if (!mbar_wait(bar.v_empty + 8 * vs, vr.ph ^ 1u, abort_flag, 2)) { record_timeout(p, abort_flag); goto done; }
+                    vr.step((uint32_t)p.v_slots);
                     SVDC_TRACE_ADD(1, p1);
                     const uint32_t vdst = v_base0 + vs * p.vslice_bytes;
                     mbar_arrive_expect_tx(bar.v_full + 8 * vs, p.vslice_bytes);
@@ -261,10 +272,11 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
                         tma_load_3d(vdst + kb * (p.gc * kTileCols * p.kb_bytes), &tm_v, bar.v_full + 8 * vs,
                                     kb * p.kb_elems, cg * kTileCols, un.b);
                     const int ce = min(cg + p.gc, un.c1);
-                    for (int c = cg; c < ce; ++c, ++it) {
-                        const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
+                    for (int c = cg; c < ce; ++c) {
+                        const uint32_t s = fr.idx;
                         SVDC_TRACE_MARK(p2);
-                        if (!mbar_wait(bar.empty + 8 * s, ph ^ 1u, abort_flag, 3)) { record_timeout(p, abort_flag); goto done; }
+                        if (!mbar_wait(bar.empty + 8 * s, fr.ph ^ 1u, abort_flag, 3)) { record_timeout(p, abort_flag); goto done; }
+                        fr.step((uint32_t)p.stages);
                         SVDC_TRACE_ADD(2, p2);
                         mbar_arrive_expect_tx(bar.full + 8 * s, kTileBytes);
                         tma_load_3d(stage0 + s * kTileBytes, &tm_r, bar.full + 8 * s, c * kTileCols, un.rt * kTileRows, un.b);
@@ -275,7 +287,8 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
     } else if (warp == 1) {
         // -------------------------------------------------------------- MMA issuer ---
         if (lane == 0) {
-            uint32_t ig = 0, ui = 0;
+            uint32_t ui = 0;
+            RingPos vr, ar;   // basis slot, accumulator stage of the next group
             const int ksteps = p.kb_elems / 16;
             for (int u = blockIdx.x; u < p.units; u += gridDim.x) {
                 const Unit un = decode_unit(p, u);
@@ -285,14 +298,16 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
                 if (!mbar_wait(bar.a_full + 8 * ab, (ui / p.a_bufs) & 1u, abort_flag, 4)) { record_timeout(p, abort_flag); goto done; }
                 SVDC_TRACE_ADD(0, m0);
                 const uint64_t a_desc0 = smem_desc_kmajor(a_base0 + ab * p.a_bytes, p.kb_bytes);
-                for (int cg = un.c0; cg < un.c1; cg += p.gc, ++ig) {
-                    const uint32_t vs = ig % p.v_slots, as = ig % p.acc_stages;
+                for (int cg = un.c0; cg < un.c1; cg += p.gc) {
+                    const uint32_t vs = vr.idx, as = ar.idx;
                     const int nsub = min(p.gc, un.c1 - cg);
                     SVDC_TRACE_MARK(m1);
-                    if (!mbar_wait(bar.v_full + 8 * vs, (ig / p.v_slots) & 1u, abort_flag, 5)) { record_timeout(p, abort_flag); goto done; }
+                    if (!mbar_wait(bar.v_full + 8 * vs, vr.ph, abort_flag, 5)) { record_timeout(p, abort_flag); goto done; }
                     SVDC_TRACE_ADD(1, m1);
                     SVDC_TRACE_MARK(m2);
-                    if (!mbar_wait(bar.acc_empty + 8 * as, ((ig / p.acc_stages) & 1u) ^ 1u, abort_flag, 6)) { record_timeout(p, abort_flag); goto done; }
+                    if (!mbar_wait(bar.acc_empty + 8 * as, ar.ph ^ 1u, abort_flag, 6)) { record_timeout(p, abort_flag); goto done; }
+                    vr.step((uint32_t)p.v_slots);
+                    ar.step((uint32_t)p.acc_stages);
                     SVDC_TRACE_ADD(2, m2);
                     tc_fence_after();
                     SVDC_TRACE_MARK(m3);
@@ -340,24 +355,26 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
         // ---------------------------------------------------------------- epilogue ---
         const int q = warp & 3, row = q * kSlabRows + lane;
         const uint32_t grp = (uint32_t)(warp - 2) >> 2;
-        uint32_t it = 0, ig = 0;
+        uint32_t it = 0;
+        RingPos fr, ar;   // R slot of chunk `it`, accumulator stage of the next group
         for (int u = blockIdx.x; u < p.units; u += gridDim.x) {
             const Unit un = decode_unit(p, u);
             if (*(volatile uint32_t *)&header_of(p, un.b)->full_steps == 0) continue;
             const int slab_row0 = un.rt * kTileRows + q * kSlabRows;
             const bool slab_live = (int64_t)slab_row0 < p.N;
-            for (int cg = un.c0; cg < un.c1; cg += p.gc, ++ig) {
-                const uint32_t as = ig % p.acc_stages, aph = (ig / p.acc_stages) & 1u;
+            for (int cg = un.c0; cg < un.c1; cg += p.gc) {
+                const uint32_t as = ar.idx, aph = ar.ph;
+                ar.step((uint32_t)p.acc_stages);
                 const int nsub = min(p.gc, un.c1 - cg);
                 const int last_own = last_own_chunk(it, nsub, grp);
                 SVDC_TRACE_MARK(e0);
                 if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar.acc_full + 8 * as, aph, abort_flag, 7))) { record_timeout(p, abort_flag); goto done; }
                 SVDC_TRACE_ADD(0, e0);
                 if (last_own < 0 && lane == 0) mbar_arrive(bar.acc_empty + 8 * as);
-                for (int j = 0; j < nsub; ++j, ++it) {
+                for (int j = 0; j < nsub; ++j, ++it, fr.step((uint32_t)p.stages)) {
                     if ((it & 1u) != grp) continue;
                     const int c = cg + j;
-                    const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
+                    const uint32_t s = fr.idx, ph = fr.ph;
                     SVDC_TRACE_MARK(e1);
                     if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar.full + 8 * s, ph, abort_flag, 8))) { record_timeout(p, abort_flag); goto done; }
                     SVDC_TRACE_ADD(1, e1);
@@ -600,6 +617,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
         // -------------------------------------------------------------- MMA issuer ---
         if (lane == 0) {
             uint32_t it = 0, iv = 0, ig = 0, ui = 0;   // F chunks, basis slices, pass-2 groups, units
+            RingPos fr, vr, ar;                        // ring positions of chunk `it`, slice `iv`, group `ig`
             const uint32_t idesc1 = idesc_bf16(kTileRows, p.k);
             const int ksteps = p.kb_elems / 16;
             const uint64_t a_desc0 = smem_desc_kmajor(a_base, p.kb_bytes);
@@ -607,12 +625,13 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                 // C of the previous unit has been read out of TMEM: a_full(ui - 1) was awaited below
                 for (int g = 0; g < G; ++g, ++iv) {                 // pass 1: C_a += F_chunk (V^T chunk)^T
                     const int cg = (g_off + g) * p.gc, ce = min(cg + p.gc, CT);
-                    const uint32_t vs = iv % p.v_slots;
+                    const uint32_t vs = vr.idx;
                     SVDC_TRACE_MARK(t0);
-                    if (!mbar_wait(bar.v_full + 8 * vs, (iv / p.v_slots) & 1u, abort_flag, 9)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
+                    if (!mbar_wait(bar.v_full + 8 * vs, vr.ph, abort_flag, 9)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
                     SVDC_TRACE_ADD(0, t0);
-                    for (int c = cg; c < ce; ++c, ++it) {
-                        const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
+                    vr.step((uint32_t)p.v_slots);
+                    for (int c = cg; c < ce; ++c, ++it, fr.step((uint32_t)p.stages)) {
+                        const uint32_t s = fr.idx, ph = fr.ph;
                         SVDC_TRACE_MARK(t1);
                         if (!mbar_wait(bar.full + 8 * s, ph, abort_flag, 10)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
                         SVDC_TRACE_ADD(1, t1);
@@ -637,13 +656,15 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                 for (int g = 0; g < G; ++g, ++iv, ++ig) {           // pass 2: acc = C (V slice)^T
                     const int cg = (g_off + G - 1 - g) * p.gc;
                     const int nsub = min(p.gc, CT - cg);
-                    const uint32_t vs = iv % p.v_slots, as = ig % p.acc_stages;
+                    const uint32_t vs = vr.idx, as = ar.idx;
                     SVDC_TRACE_MARK(t4);
-                    if (!mbar_wait(bar.v_full + 8 * vs, (iv / p.v_slots) & 1u, abort_flag, 12)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
+                    if (!mbar_wait(bar.v_full + 8 * vs, vr.ph, abort_flag, 12)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
                     SVDC_TRACE_ADD(4, t4);
                     SVDC_TRACE_MARK(t5);
-                    if (!mbar_wait(bar.acc_empty + 8 * as, ((ig / p.acc_stages) & 1u) ^ 1u, abort_flag, 13)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
+                    if (!mbar_wait(bar.acc_empty + 8 * as, ar.ph ^ 1u, abort_flag, 13)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
                     SVDC_TRACE_ADD(5, t5);
+                    vr.step((uint32_t)p.v_slots);
+                    ar.step((uint32_t)p.acc_stages);
                     tc_fence_after();
                     SVDC_TRACE_MARK(t6);
                     const uint32_t idesc = idesc_bf16(kTileRows, nsub * kTileCols);
@@ -667,10 +688,9 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                     // satisfied by the phase before a skipped one), and the slot must not be reused
                     // before it has: it waits for the group's chunks here, after the MMAs are on their
                     // way, and its arrival is one of the five that free the slot.
-                    for (int j = 0; j < nsub; ++j, ++it) {
-                        const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                        if (!mbar_wait(bar.full + 8 * s, ph, abort_flag, 19)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
-                        mbar_arrive(bar.empty + 8 * s);
+                    for (int j = 0; j < nsub; ++j, ++it, fr.step((uint32_t)p.stages)) {
+                        if (!mbar_wait(bar.full + 8 * fr.idx, fr.ph, abort_flag, 19)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
+                        mbar_arrive(bar.empty + 8 * fr.idx);
                     }
                 }
                 mma_commit(p2_done);
@@ -686,6 +706,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
         const uint32_t chat_row_bytes = p.k >= 32 ? 128u : (uint32_t)p.k * 4u;
         const int nblk = (p.k + 31) / 32;
         uint32_t it = 0, ig = 0, ui = 0, nchat = 0;   // F chunks, pass-2 groups, units, Chat tiles consumed
+        RingPos fr, ar;                               // ring positions of chunk `it`, group `ig`
         int prev_slot = -1;                           // slot whose slab store may still be reading
         const bool defer_release = p.stages >= 4;
 
@@ -851,19 +872,21 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
             const int slab_row0 = un.rt * kTileRows + q * kSlabRows;
             const bool slab_live = (int64_t)slab_row0 < p.N;
             it += CTm;   // pass-1 slots are consumed by the MMA warp alone
+            fr.skip((uint32_t)CTm, (uint32_t)p.stages);
             for (int g = 0; g < G; ++g, ++ig) {
                 const int cg = (g_off + G - 1 - g) * p.gc;
                 const int nsub = min(p.gc, CT - cg);
-                const uint32_t as = ig % p.acc_stages, aph = (ig / p.acc_stages) & 1u;
+                const uint32_t as = ar.idx, aph = ar.ph;
+                ar.step((uint32_t)p.acc_stages);
                 const int last_own = last_own_chunk(it, nsub, grp);
                 SVDC_TRACE_MARK(e3);
                 if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar.acc_full + 8 * as, aph, abort_flag, 16))) { record_timeout(p, abort_flag, it, ig, ui); goto done; }
                 SVDC_TRACE_ADD(3, e3);
                 if (last_own < 0 && lane == 0) mbar_arrive(bar.acc_empty + 8 * as);
-                for (int j = 0; j < nsub; ++j, ++it) {
+                for (int j = 0; j < nsub; ++j, ++it, fr.step((uint32_t)p.stages)) {
                     if ((it & 1u) != grp) continue;
                     const int c = cg + j;
-                    const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
+                    const uint32_t s = fr.idx, ph = fr.ph;
                     SVDC_TRACE_MARK(e4);
                     if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar.full + 8 * s, ph, abort_flag, 17))) { record_timeout(p, abort_flag, it, ig, ui); goto done; }
                     SVDC_TRACE_ADD(4, e4);
