@@ -487,6 +487,20 @@ __device__ __forceinline__ void pack_split8(const float *v, uint4 &hi, uint4 &lo
     lo = make_uint4(l[0], l[1], l[2], l[3]);
 }
 
+// 32-byte stores: a thread of the C job owns a whole row, so every store instruction touches 32
+// different lines -- the fewer and wider they are, the less time the job spends in the
+// load-store unit
+__device__ __forceinline__ void stg256(float *dst, const float *v) {
+    asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "f"(v[0]), "f"(v[1]), "f"(v[2]),
+                 "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7])
+                 : "memory");
+}
+__device__ __forceinline__ void stg256(void *dst, uint4 a, uint4 b) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(a.x), "r"(a.y), "r"(a.z),
+                 "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w)
+                 : "memory");
+}
+
 template <bool kClusterSplit>
 __global__ void __launch_bounds__(kThreadsFull, 1)
 umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant__ CUtensorMap tm_vt,
@@ -505,6 +519,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
     // cluster mode: peer_ready (the peer's A region may be written), recv_full (the peer's
     // partial C has arrived in mine)
     const uint32_t chat_full = bar.a_full + 8, p2_done = bar.c_done, peer_ready = bar.a_empty, recv_full = bar.a_empty + 8;
+    const uint32_t c_read = peer_ready;   // split C job (never with a cluster): staged inputs read by all 256 threads
     uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
     volatile int *abort_flag = reinterpret_cast<volatile int *>(gen_base + (bar.abort_flag - base));
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(gen_base + (bar.tmem_slot - base));
@@ -524,6 +539,9 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
     const int c_first = g_off * p.gc;
     const int CTm = min(CT, (g_off + G) * p.gc) - c_first;                   // this CTA's chunks per pass
     const uint32_t a_part = p.k >= 64 ? kBlk32Bytes : p.a_half_bytes;   // hi -> lo distance
+    // From k = 64 on, both epilogue groups share the C job: of every 64-column block of C the C
+    // warps (6..9) take the lower 32 columns, warps 2..5 the upper 32.
+    const bool c_split = !kClusterSplit && p.k >= 64;
     const uint32_t a_kb = 2u * kBlk32Bytes;                             // K-block distance (k >= 64)
 
     if (threadIdx.x == 0) {
@@ -532,11 +550,11 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
         for (int s = 0; s < p.stages; ++s) { mbar_init(bar.full + 8 * s, 1); mbar_init(bar.empty + 8 * s, 5); }
         for (int s = 0; s < p.acc_stages; ++s) { mbar_init(bar.acc_full + 8 * s, 1); mbar_init(bar.acc_empty + 8 * s, 8); }
         for (int s = 0; s < p.v_slots; ++s) { mbar_init(bar.v_full + 8 * s, 1); mbar_init(bar.v_empty + 8 * s, 1); }
-        mbar_init(bar.a_full, 128);
+        mbar_init(bar.a_full, c_split ? 256 : 128);
         mbar_init(chat_full, 1);
         mbar_init(bar.c_full, 1);
         mbar_init(p2_done, 1);
-        mbar_init(peer_ready, 1);
+        mbar_init(peer_ready, c_split ? 256 : 1);   // c_read when the C job is split
         mbar_init(recv_full, 128);
         *abort_flag = 0;
         fence_barrier_init();
@@ -705,7 +723,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
         const float beta = p.beta, omb = 1.0f - p.beta;
         const uint32_t chat_row_bytes = p.k >= 32 ? 128u : (uint32_t)p.k * 4u;
         const int nblk = (p.k + 31) / 32;
-        uint32_t it = 0, ig = 0, ui = 0, nchat = 0;   // F chunks, pass-2 groups, units, Chat tiles consumed
+        uint32_t it = 0, ig = 0, ui = 0, nchat = 0, ncread = 0;   // F chunks, pass-2 groups, units, Chat tiles consumed, c_read phases
         RingPos fr, ar;                               // ring positions of chunk `it`, group `ig`
         int prev_slot = -1;                           // slot whose slab store may still be reading
         const bool defer_release = p.stages >= 4;
@@ -721,7 +739,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
         }
         for (int u = cid; u < p.units; u += nclusters, ++ui) {
             const Unit un = decode_unit(p, u);
-            if (c_warp) {
+            if (c_warp || c_split) {
                 // ---- C job: TMEM -> EMA -> Chat, split-bf16 A operand (+ the state's operand copy)
                 StateHeader *hdr = header_of(p, un.b);
                 const bool first = *(volatile uint32_t *)&hdr->full_steps == 0;
@@ -777,13 +795,24 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                     const uint32_t hi_row = a_base + (uint32_t)kb * a_kb + (uint32_t)row * p.kb_bytes;
                     const uint32_t lo_row = hi_row + a_part;
                     const int halves = p.k >= 64 ? 2 : 1;
-                    float prevB[32];
-                    if (!first && halves == 2) load_row32(stB, (uint32_t)row, chat_row_bytes, 32, prevB);
+                    // split job: this warp's half only; its staged input is read, and the partner warp's
+                    // too, before either writes operand rows over them
+                    const int h_lo = c_split ? (c_warp ? 0 : 1) : 0, h_hi = c_split ? h_lo + 1 : halves;
+                    float prevB[32];   // staged Chat of the upper half -- of this thread's half when the job is split
+                    if (!first && halves == 2) load_row32(c_split && h_lo == 0 ? stA : stB, (uint32_t)row, chat_row_bytes, 32, prevB);
+                    if constexpr (!kClusterSplit) {
+                        if (c_split) {
+                            // (all 256 threads meet: a bounded wait on an mbarrier, like every other wait here)
+                            mbar_arrive(c_read);
+                            if (!__all_sync(0xFFFFFFFFu, mbar_wait(c_read, ncread & 1u, abort_flag, 22))) { record_timeout(p, abort_flag, it, ig, ui); goto done; }
+                            ++ncread;
+                        }
+                    }
                     // cluster mode: the peer's partial sits where this row's hi / lo operand rows go
                     // (the staged Chat has a buffer of its own then); read the lo half's block first
                     float recvB[kClusterSplit ? 32 : 1];
                     if constexpr (kClusterSplit) load_row32(lo_row, (uint32_t)row, 128u, 32, recvB);
-                    for (int h = 0; h < halves; ++h) {
+                    for (int h = h_lo; h < h_hi; ++h) {
                         const int col0 = kb * 64 + h * 32;
                         const int ncols = p.k - col0 < 32 ? p.k - col0 : 32;
                         float cs[32];
@@ -810,7 +839,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
 #pragma unroll
                             for (int i = 0; i < 32; ++i) ch[i] = cs[i];
                         } else {
-                            if (h == 0) load_row32(stA, (uint32_t)row, chat_row_bytes, ncols, ch);
+                            if (h == 0 && !c_split) load_row32(stA, (uint32_t)row, chat_row_bytes, ncols, ch);
                             else {
 #pragma unroll
                                 for (int i = 0; i < 32; ++i) ch[i] = prevB[i];
@@ -829,36 +858,39 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                                 sts128(lo_row + chunk, lo);
                             }
                         }
+                        // The operand is what pass 2 waits for: once this thread's last piece of it is
+                        // written, say so, and only then send the coefficient arrays on their way -- under
+                        // a saturated memory system the stores below take microseconds to be accepted.
+                        if (kb == nkb64 - 1 && h == h_hi - 1) {
+                            tc_fence_before();
+                            fence_proxy_async();
+                            mbar_arrive(bar.a_full);
+                            SVDC_TRACE_ADD(2, c2);
+                        }
                         if (row_live) {
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) {
-                                if (i * 4 < ncols) {
-                                    *reinterpret_cast<float4 *>(chat_g + col0 + 4 * i) =
-                                        make_float4(ch[4 * i], ch[4 * i + 1], ch[4 * i + 2], ch[4 * i + 3]);
-                                    if (cout_g)
-                                        *reinterpret_cast<float4 *>(cout_g + col0 + 4 * i) =
-                                            make_float4(cs[4 * i], cs[4 * i + 1], cs[4 * i + 2], cs[4 * i + 3]);
+                            for (int i = 0; i < 4; ++i) {
+                                if (i * 8 < ncols) {
+                                    stg256(chat_g + col0 + 8 * i, ch + 8 * i);
+                                    if (cout_g) stg256(cout_g + col0 + 8 * i, cs + 8 * i);
                                 }
                             }
                             // ... while the state keeps the split of the new Chat
                             __nv_bfloat16 *ohi = reinterpret_cast<__nv_bfloat16 *>(st_b + p.ophi_off) + n * p.k + col0;
                             __nv_bfloat16 *olo = reinterpret_cast<__nv_bfloat16 *>(st_b + p.oplo_off) + n * p.k + col0;
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                if (i * 8 < ncols) {
-                                    uint4 hi, lo;
-                                    pack_split8(ch + 8 * i, hi, lo);
-                                    *reinterpret_cast<uint4 *>(ohi + 8 * i) = hi;
-                                    *reinterpret_cast<uint4 *>(olo + 8 * i) = lo;
+                            for (int i = 0; i < 2; ++i) {
+                                if (i * 16 < ncols) {
+                                    uint4 hi0, lo0, hi1, lo1;
+                                    pack_split8(ch + 16 * i, hi0, lo0);
+                                    pack_split8(ch + 16 * i + 8, hi1, lo1);
+                                    stg256(ohi + 16 * i, hi0, hi1);
+                                    stg256(olo + 16 * i, lo0, lo1);
                                 }
                             }
                         }
                     }
                 }
-                tc_fence_before();
-                fence_proxy_async();
-                mbar_arrive(bar.a_full);
-                SVDC_TRACE_ADD(2, c2);
                 // count this unit; the last unit of a block to get here counts the full step
                 if (issuer && crank == 0) {
                     const uint32_t prev = atomicAdd(&hdr->done, 1u);
