@@ -30,7 +30,7 @@ constexpr int kTileCols = 64;       // columns of D per stage (MMA N in the reco
 constexpr int kTileBytes = kTileRows * kTileCols * 2;   // 16 KB
 constexpr int kAccStages = 4;       // TMEM accumulator ring (64 fp32 columns each)
 constexpr int kMaxStages = 12;
-constexpr int kMaxVSlots = 2;
+constexpr int kMaxVSlots = 4;
 constexpr int kMaxABufs = 2;
 
 struct UmmaParams {
@@ -442,9 +442,12 @@ done:
 // A unit is one 128-row tile of one block.
 //   Pass 1 streams the tile's F in 64-column chunks and accumulates C (128 x k, fp32) in
 //     TMEM: A = F chunk, B = matching columns of V_k^T.
-//   The C warps read C from TMEM, apply the EMA against the previous Chat (staged by TMA in
-//     the A-operand region and converted in place), write Chat, and leave C as a split-bf16
-//     A operand in shared memory -- which also goes out, as it is, as the state's operand copy.
+//   The C job reads C from TMEM, applies the EMA against the previous Chat, writes Chat, its
+//     split-bf16 copy for the cached step and C_out, and leaves C itself as a split-bf16 A
+//     operand: from k = 64 on in tensor memory, over the columns of C (kTmemA: both epilogue
+//     groups share the job, the previous Chat comes through registers, and all of shared memory
+//     goes to the rings); below that, and in a cluster, in a shared-memory region that also
+//     stages the previous Chat by TMA (warps 6..9 alone).
 //   Pass 2 streams the same F chunks again, last group first (the most recently read ones
 //     are the likeliest to sit in L2), with V_k slices of gc*64 rows: C V_k^T per group in
 //     TMEM, and the epilogue stores R = F - C V_k^T through TMA.
@@ -453,9 +456,9 @@ done:
 // slice one group ahead of the F chunks that go with it.
 //
 // Warp roles (352 threads): 0 = TMA producer of the F chunks, 10 = TMA producer of the basis
-// slices, 1 = MMA issuer (+ TMEM owner), 2..5 = epilogue group 0, 6..9 = C warps, which turn
-// into epilogue group 1 once the A operand is written (pass 2 cannot start before that, so
-// the two jobs never overlap).
+// slices, 1 = MMA issuer (+ TMEM owner), 2..5 and 6..9 = the two epilogue groups of pass 2,
+// which first do the C job (pass 2 cannot start before the operand is written, so the two
+// jobs never overlap).
 // ======================================================================================
 constexpr int kThreadsFull = 352;
 constexpr int kFullVWarp = 10;   // second TMA producer (basis slices); warps 2..9 are the epilogue
@@ -501,7 +504,7 @@ __device__ __forceinline__ void stg256(void *dst, uint4 a, uint4 b) {
                  : "memory");
 }
 
-template <bool kClusterSplit>
+template <bool kClusterSplit, bool kTmemA>
 __global__ void __launch_bounds__(kThreadsFull, 1)
 umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant__ CUtensorMap tm_vt,
                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_rout,
@@ -519,7 +522,6 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
     // cluster mode: peer_ready (the peer's A region may be written), recv_full (the peer's
     // partial C has arrived in mine)
     const uint32_t chat_full = bar.a_full + 8, p2_done = bar.c_done, peer_ready = bar.a_empty, recv_full = bar.a_empty + 8;
-    const uint32_t c_read = peer_ready;   // split C job (never with a cluster): staged inputs read by all 256 threads
     uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
     volatile int *abort_flag = reinterpret_cast<volatile int *>(gen_base + (bar.abort_flag - base));
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(gen_base + (bar.tmem_slot - base));
@@ -539,9 +541,11 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
     const int c_first = g_off * p.gc;
     const int CTm = min(CT, (g_off + G) * p.gc) - c_first;                   // this CTA's chunks per pass
     const uint32_t a_part = p.k >= 64 ? kBlk32Bytes : p.a_half_bytes;   // hi -> lo distance
-    // From k = 64 on, both epilogue groups share the C job: of every 64-column block of C the C
-    // warps (6..9) take the lower 32 columns, warps 2..5 the upper 32.
-    const bool c_split = !kClusterSplit && p.k >= 64;
+    // From k = 64 on (and without a cluster) the A operand of pass 2 lives in tensor memory, over
+    // C itself, and both epilogue groups share the C job; below that it is staged in shared memory.
+    // (Each variant is an instantiation of its own: compiled together, the two C jobs spill.)
+    constexpr bool c_split = kTmemA;
+    static_assert(!(kClusterSplit && kTmemA), "the cluster exchange uses the shared-memory operand region");
     const uint32_t a_kb = 2u * kBlk32Bytes;                             // K-block distance (k >= 64)
 
     if (threadIdx.x == 0) {
@@ -554,7 +558,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
         mbar_init(chat_full, 1);
         mbar_init(bar.c_full, 1);
         mbar_init(p2_done, 1);
-        mbar_init(peer_ready, c_split ? 256 : 1);   // c_read when the C job is split
+        mbar_init(peer_ready, 1);
         mbar_init(recv_full, 128);
         *abort_flag = 0;
         fence_barrier_init();
@@ -694,7 +698,11 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                             const uint64_t ad = a_desc0 + ((part * a_part + kb * a_kb) >> 4);
                             const uint64_t vd = v_desc0 + ((kb * (p.gc * kTileCols * p.kb_bytes)) >> 4);
                             for (int ks = 0; ks < ksteps; ++ks) {
-                                mma_bf16_ss(d_tmem, ad + 2 * ks, vd + 2 * ks, idesc, acc);
+                                if constexpr (c_split)   // operand in TMEM: 64-column block kb, half ks / 2, hi or lo words, K step
+                                    mma_bf16_ts(d_tmem, tmem_base + (uint32_t)(kb * 64 + (ks >> 1) * 32 + part * 16 + (ks & 1) * 8),
+                                                vd + 2 * ks, idesc, acc);
+                                else
+                                    mma_bf16_ss(d_tmem, ad + 2 * ks, vd + 2 * ks, idesc, acc);
                                 acc = 1;
                             }
                         }
@@ -723,7 +731,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
         const float beta = p.beta, omb = 1.0f - p.beta;
         const uint32_t chat_row_bytes = p.k >= 32 ? 128u : (uint32_t)p.k * 4u;
         const int nblk = (p.k + 31) / 32;
-        uint32_t it = 0, ig = 0, ui = 0, nchat = 0, ncread = 0;   // F chunks, pass-2 groups, units, Chat tiles consumed, c_read phases
+        uint32_t it = 0, ig = 0, ui = 0, nchat = 0;   // F chunks, pass-2 groups, units, Chat tiles consumed
         RingPos fr, ar;                               // ring positions of chunk `it`, group `ig`
         int prev_slot = -1;                           // slot whose slab store may still be reading
         const bool defer_release = p.stages >= 4;
@@ -733,13 +741,107 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
             for (int b = 0; b < nblk; ++b)
                 tma_load_3d(chat_base + b * kBlk32Bytes, &tm_chat, chat_full, b * 32, x.rt * kTileRows, x.b);
         };
-        if (issuer && cid < p.units) {
+        if (issuer && cid < p.units && !c_split) {
             const Unit x = decode_unit(p, cid);
             if (*(volatile uint32_t *)&header_of(p, x.b)->full_steps != 0) request_chat(x);
         }
         for (int u = cid; u < p.units; u += nclusters, ++ui) {
             const Unit un = decode_unit(p, u);
-            if (c_warp || c_split) {
+            if constexpr (c_split) {
+                // ---- C job, operand in tensor memory (k >= 64): both epilogue groups take part.  Of
+                // every 64-column block of C, a thread of warps 6..9 owns the lower 32 columns of its
+                // row and a thread of warps 2..5 the upper 32: it reads them from TMEM, applies the EMA
+                // against the previous Chat (prefetched into registers while pass 1 ran), and writes the
+                // split-bf16 pair back over the very columns it has read -- 16 columns of hi words,
+                // then 16 of lo words (two bf16 per 32-bit column) -- which is where the MMAs of pass 2
+                // take their A operand from.  No staging, no shared memory, nobody else's columns.
+                StateHeader *hdr = header_of(p, un.b);
+                const bool first = *(volatile uint32_t *)&hdr->full_steps == 0;
+                const int h = c_warp ? 0 : 1;
+                const int64_t n = (int64_t)un.rt * kTileRows + row;
+                const bool row_live = n < p.N;
+                char *st_b = p.state + (size_t)un.b * p.state_stride;
+                float *chat_g = reinterpret_cast<float *>(st_b + p.chat_off) + n * p.k + h * 32;
+                float *cout_g = p.C_out ? reinterpret_cast<float *>((char *)p.C_out + (size_t)un.b * p.C_stride) + n * p.k + h * 32
+                                        : nullptr;
+                __nv_bfloat16 *ohi = reinterpret_cast<__nv_bfloat16 *>(st_b + p.ophi_off) + n * p.k + h * 32;
+                __nv_bfloat16 *olo = reinterpret_cast<__nv_bfloat16 *>(st_b + p.oplo_off) + n * p.k + h * 32;
+                auto load_prev = [&](int kb, float (&pv)[32]) {
+                    if (!first && row_live) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const float4 t = *reinterpret_cast<const float4 *>(chat_g + kb * 64 + 4 * i);
+                            pv[4 * i] = t.x; pv[4 * i + 1] = t.y; pv[4 * i + 2] = t.z; pv[4 * i + 3] = t.w;
+                        }
+                    }
+                };
+                float prev0[32];   // previous Chat of the first K block: on its way while pass 1 runs
+                load_prev(0, prev0);
+                SVDC_TRACE_MARK(c1);
+                if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar.c_full, ui & 1u, abort_flag, 15))) { record_timeout(p, abort_flag, it, ig, ui); goto done; }
+                SVDC_TRACE_ADD(1, c1);
+                tc_fence_after();
+                SVDC_TRACE_MARK(c2);
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * 32);
+                auto k_block = [&](int kb, float (&pv)[32]) {
+                    uint32_t w[32];
+                    tmem_ld_32x32(taddr + kb * 64, w);
+                    tmem_wait_ld();
+                    float cs[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) cs[i] = __uint_as_float(w[i]);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {   // hi words of columns 8i..8i+7 -> w[4i..], lo words -> w[16+4i..]
+                        uint4 hi, lo;
+                        pack_split8(cs + 8 * i, hi, lo);
+                        w[4 * i] = hi.x; w[4 * i + 1] = hi.y; w[4 * i + 2] = hi.z; w[4 * i + 3] = hi.w;
+                        w[16 + 4 * i] = lo.x; w[16 + 4 * i + 1] = lo.y; w[16 + 4 * i + 2] = lo.z; w[16 + 4 * i + 3] = lo.w;
+                    }
+                    tmem_st_32x32(taddr + kb * 64, w);
+                    if (kb == p.nkb - 1) {   // the operand is what pass 2 waits for: announce it before the stores below
+                        tmem_wait_st();
+                        tc_fence_before();
+                        mbar_arrive(bar.a_full);
+                        SVDC_TRACE_ADD(2, c2);
+                    }
+                    if (row_live) {
+                        if (!first) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) pv[i] = fmaf(beta, pv[i], omb * cs[i]);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) pv[i] = cs[i];
+                        }
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            stg256(chat_g + kb * 64 + 8 * i, pv + 8 * i);
+                            if (cout_g) stg256(cout_g + kb * 64 + 8 * i, cs + 8 * i);
+                        }
+#pragma unroll
+                        for (int i = 0; i < 2; ++i) {   // the state keeps the split of the new Chat
+                            uint4 hi0, lo0, hi1, lo1;
+                            pack_split8(pv + 16 * i, hi0, lo0);
+                            pack_split8(pv + 16 * i + 8, hi1, lo1);
+                            stg256(ohi + kb * 64 + 16 * i, hi0, hi1);
+                            stg256(olo + kb * 64 + 16 * i, lo0, lo1);
+                        }
+                    }
+                };
+                for (int kb = 0; kb < p.nkb; ++kb) {
+                    // wider ranks: the previous Chat of the later blocks is fetched as it is needed -- the
+                    // operand does not wait for it, only this thread's own stores do
+                    if (kb > 0) load_prev(kb, prev0);
+                    k_block(kb, prev0);
+                }
+                // count this unit; the last unit of a block to get here counts the full step
+                if (issuer) {
+                    const uint32_t prevc = atomicAdd(&hdr->done, 1u);
+                    if (prevc == (uint32_t)p.row_tiles - 1u) {
+                        hdr->done = 0;
+                        hdr->full_steps = hdr->full_steps + 1;
+                    }
+                }
+            } else if (c_warp) {   // (discarded statement of the if constexpr above when the operand is in TMEM)
                 // ---- C job: TMEM -> EMA -> Chat, split-bf16 A operand (+ the state's operand copy)
                 StateHeader *hdr = header_of(p, un.b);
                 const bool first = *(volatile uint32_t *)&hdr->full_steps == 0;
@@ -795,24 +897,13 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                     const uint32_t hi_row = a_base + (uint32_t)kb * a_kb + (uint32_t)row * p.kb_bytes;
                     const uint32_t lo_row = hi_row + a_part;
                     const int halves = p.k >= 64 ? 2 : 1;
-                    // split job: this warp's half only; its staged input is read, and the partner warp's
-                    // too, before either writes operand rows over them
-                    const int h_lo = c_split ? (c_warp ? 0 : 1) : 0, h_hi = c_split ? h_lo + 1 : halves;
-                    float prevB[32];   // staged Chat of the upper half -- of this thread's half when the job is split
-                    if (!first && halves == 2) load_row32(c_split && h_lo == 0 ? stA : stB, (uint32_t)row, chat_row_bytes, 32, prevB);
-                    if constexpr (!kClusterSplit) {
-                        if (c_split) {
-                            // (all 256 threads meet: a bounded wait on an mbarrier, like every other wait here)
-                            mbar_arrive(c_read);
-                            if (!__all_sync(0xFFFFFFFFu, mbar_wait(c_read, ncread & 1u, abort_flag, 22))) { record_timeout(p, abort_flag, it, ig, ui); goto done; }
-                            ++ncread;
-                        }
-                    }
+                    float prevB[32];
+                    if (!first && halves == 2) load_row32(stB, (uint32_t)row, chat_row_bytes, 32, prevB);
                     // cluster mode: the peer's partial sits where this row's hi / lo operand rows go
                     // (the staged Chat has a buffer of its own then); read the lo half's block first
                     float recvB[kClusterSplit ? 32 : 1];
                     if constexpr (kClusterSplit) load_row32(lo_row, (uint32_t)row, 128u, 32, recvB);
-                    for (int h = h_lo; h < h_hi; ++h) {
+                    for (int h = 0; h < halves; ++h) {
                         const int col0 = kb * 64 + h * 32;
                         const int ncols = p.k - col0 < 32 ? p.k - col0 : 32;
                         float cs[32];
@@ -839,7 +930,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
 #pragma unroll
                             for (int i = 0; i < 32; ++i) ch[i] = cs[i];
                         } else {
-                            if (h == 0 && !c_split) load_row32(stA, (uint32_t)row, chat_row_bytes, ncols, ch);
+                            if (h == 0) load_row32(stA, (uint32_t)row, chat_row_bytes, ncols, ch);
                             else {
 #pragma unroll
                                 for (int i = 0; i < 32; ++i) ch[i] = prevB[i];
@@ -858,39 +949,36 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                                 sts128(lo_row + chunk, lo);
                             }
                         }
-                        // The operand is what pass 2 waits for: once this thread's last piece of it is
-                        // written, say so, and only then send the coefficient arrays on their way -- under
-                        // a saturated memory system the stores below take microseconds to be accepted.
-                        if (kb == nkb64 - 1 && h == h_hi - 1) {
-                            tc_fence_before();
-                            fence_proxy_async();
-                            mbar_arrive(bar.a_full);
-                            SVDC_TRACE_ADD(2, c2);
-                        }
                         if (row_live) {
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                if (i * 8 < ncols) {
-                                    stg256(chat_g + col0 + 8 * i, ch + 8 * i);
-                                    if (cout_g) stg256(cout_g + col0 + 8 * i, cs + 8 * i);
+                            for (int i = 0; i < 8; ++i) {
+                                if (i * 4 < ncols) {
+                                    *reinterpret_cast<float4 *>(chat_g + col0 + 4 * i) =
+                                        make_float4(ch[4 * i], ch[4 * i + 1], ch[4 * i + 2], ch[4 * i + 3]);
+                                    if (cout_g)
+                                        *reinterpret_cast<float4 *>(cout_g + col0 + 4 * i) =
+                                            make_float4(cs[4 * i], cs[4 * i + 1], cs[4 * i + 2], cs[4 * i + 3]);
                                 }
                             }
                             // ... while the state keeps the split of the new Chat
                             __nv_bfloat16 *ohi = reinterpret_cast<__nv_bfloat16 *>(st_b + p.ophi_off) + n * p.k + col0;
                             __nv_bfloat16 *olo = reinterpret_cast<__nv_bfloat16 *>(st_b + p.oplo_off) + n * p.k + col0;
 #pragma unroll
-                            for (int i = 0; i < 2; ++i) {
-                                if (i * 16 < ncols) {
-                                    uint4 hi0, lo0, hi1, lo1;
-                                    pack_split8(ch + 16 * i, hi0, lo0);
-                                    pack_split8(ch + 16 * i + 8, hi1, lo1);
-                                    stg256(ohi + 16 * i, hi0, hi1);
-                                    stg256(olo + 16 * i, lo0, lo1);
+                            for (int i = 0; i < 4; ++i) {
+                                if (i * 8 < ncols) {
+                                    uint4 hi, lo;
+                                    pack_split8(ch + 8 * i, hi, lo);
+                                    *reinterpret_cast<uint4 *>(ohi + 8 * i) = hi;
+                                    *reinterpret_cast<uint4 *>(olo + 8 * i) = lo;
                                 }
                             }
                         }
                     }
                 }
+                tc_fence_before();
+                fence_proxy_async();
+                mbar_arrive(bar.a_full);
+                SVDC_TRACE_ADD(2, c2);
                 // count this unit; the last unit of a block to get here counts the full step
                 if (issuer && crank == 0) {
                     const uint32_t prev = atomicAdd(&hdr->done, 1u);
@@ -975,7 +1063,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
             if (issuer) {
                 const int un_next = u + nclusters;
                 const bool ok = mbar_wait(p2_done, ui & 1u, abort_flag, 18);
-                if (ok && un_next < p.units) {
+                if (ok && un_next < p.units && !c_split) {
                     const Unit x = decode_unit(p, un_next);
                     if (*(volatile uint32_t *)&header_of(p, x.b)->full_steps != 0) request_chat(x);
                 }
@@ -1640,7 +1728,7 @@ void fill_groups(const StepArgs &a, UmmaParams &p) {
     p.acc_cols = p.gc * kTileCols;
     p.acc_stages = 512 / p.acc_cols < kAccStages ? 512 / p.acc_cols : kAccStages;
     p.vslice_bytes = (uint32_t)p.gc * kTileCols * a.k * 2;
-    p.v_slots = kMaxVSlots;
+    p.v_slots = 2;
 }
 
 // Full step: shared memory = A operand region (+ Chat staging when k < 64) | basis ring | F ring | barriers.
@@ -1653,18 +1741,28 @@ bool fill_full(const StepArgs &a, UmmaParams &p, int cluster = 1) {
     p.acc_cols = p.gc * kTileCols;
     p.acc_stages = (512 - a.k) / p.acc_cols < kAccStages ? (512 - a.k) / p.acc_cols : kAccStages;
     p.vslice_bytes = (uint32_t)p.gc * kTileCols * a.k * 2;
-    // the staged previous Chat shares the A region (converted in place) when k >= 64, unless
-    // the region doubles as the receive buffer of a cluster's exchange
-    const bool in_place = a.k >= 64 && cluster == 1;
-    p.chat_stage_off = in_place ? 0u : p.a_bytes;
-    p.a_region_bytes = p.a_bytes + (in_place ? 0u : (uint32_t)kTileRows * a.k * 4u);
+    // From k = 64 on the A operand lives in tensor memory (the kernel's c_split) and the previous
+    // Chat comes through registers: no A region at all, and the shared memory goes to the rings --
+    // a third basis slot first (a slice arrives 2000-3000 cycles after its request under load, a
+    // group of MMAs lasts ~1000), a fourth if it costs no F slot.  Below k = 64, and in a cluster,
+    // the operand and the staged Chat share a region of shared memory.
+    const bool a_tmem = a.k >= 64 && cluster == 1;
+    p.chat_stage_off = a_tmem ? 0u : p.a_bytes;
+    p.a_region_bytes = a_tmem ? 0u : p.a_bytes + (uint32_t)kTileRows * a.k * 4u;
     p.a_region_bytes = (p.a_region_bytes + 1023u) & ~1023u;
     const size_t avail = kSmemBudget - 1024 /*alignment*/ - kBarBytes - 64;
-    const size_t fixed = (size_t)p.a_region_bytes + (size_t)p.v_slots * p.vslice_bytes;
-    if (fixed + 2 * (size_t)kTileBytes > avail) return false;
-    p.stages = (int)((avail - fixed) / kTileBytes);
-    if (p.stages > kMaxStages) p.stages = kMaxStages;
-    p.stages &= ~1;   // even: a slot then always serves the same epilogue group (chunk parity)
+    auto stages_for = [&](int v_slots) {
+        const size_t fixed = (size_t)p.a_region_bytes + (size_t)v_slots * p.vslice_bytes;
+        if (fixed + 2 * (size_t)kTileBytes > avail) return 0;
+        int st = (int)((avail - fixed) / kTileBytes);
+        if (st > kMaxStages) st = kMaxStages;
+        return st & ~1;   // even: a slot then always serves the same epilogue group (chunk parity)
+    };
+    p.v_slots = 2;
+    if (a_tmem && stages_for(3) >= 8) p.v_slots = 3;
+    if (a_tmem && p.v_slots == 3 && stages_for(4) == stages_for(3)) p.v_slots = 4;
+    p.stages = stages_for(p.v_slots);
+    if (p.stages < 2) return false;
     p.a_bufs = 1;
     return true;
 }
@@ -1822,7 +1920,7 @@ int max_full_clusters(size_t smem) {
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, umma_full_kernel<true>, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+    if (cudaOccupancyMaxActiveClusters(&n, umma_full_kernel<true, false>, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
     cached = n;
     return n;
 }
@@ -1878,10 +1976,13 @@ int umma_full_step(const StepArgs &a, cudaStream_t s) {
 
     static bool attr_set = false;
     if (!attr_set) {
-        int rc0 = record_cuda(cudaFuncSetAttribute(umma_full_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        int rc0 = record_cuda(cudaFuncSetAttribute(umma_full_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                    (int)kSmemBudget));
         if (rc0) return rc0;
-        rc0 = record_cuda(cudaFuncSetAttribute(umma_full_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        rc0 = record_cuda(cudaFuncSetAttribute(umma_full_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               (int)kSmemBudget));
+        if (rc0) return rc0;
+        rc0 = record_cuda(cudaFuncSetAttribute(umma_full_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                (int)kSmemBudget));
         if (rc0) return rc0;
         attr_set = true;
@@ -1935,12 +2036,15 @@ int umma_full_step(const StepArgs &a, cudaStream_t s) {
         attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
         cfg.attrs = &attr;
         cfg.numAttrs = 1;
-        rc = record_cuda(cudaLaunchKernelEx(&cfg, umma_full_kernel<true>, tm_f, tm_vt, tm_v, tm_rout, tm_chat, p));
+        rc = record_cuda(cudaLaunchKernelEx(&cfg, umma_full_kernel<true, false>, tm_f, tm_vt, tm_v, tm_rout, tm_chat, p));
         count_launch();
         return rc ? rc : check_last_launch();
     }
     const int grid = p.units < num_sms() ? p.units : num_sms();
-    umma_full_kernel<false><<<grid, kThreadsFull, smem, s>>>(tm_f, tm_vt, tm_v, tm_rout, tm_chat, p);
+    if (a.k >= 64)   // operand in tensor memory (fill_full has sized the rings for it)
+        umma_full_kernel<false, true><<<grid, kThreadsFull, smem, s>>>(tm_f, tm_vt, tm_v, tm_rout, tm_chat, p);
+    else
+        umma_full_kernel<false, false><<<grid, kThreadsFull, smem, s>>>(tm_f, tm_vt, tm_v, tm_rout, tm_chat, p);
     count_launch();
     return check_last_launch();
 }
