@@ -735,6 +735,9 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
         RingPos fr, ar;                               // ring positions of chunk `it`, group `ig`
         int prev_slot = -1;                           // slot whose slab store may still be reading
         const bool defer_release = p.stages >= 4;
+        // R is not read again by this step: its lines are the first to go, which leaves more of L2 to
+        // the F tiles waiting for their second pass
+        const uint64_t pol_store = policy_evict_first();
 
         auto request_chat = [&](const Unit &x) {   // previous Chat of unit x -> staging, by TMA
             mbar_arrive_expect_tx(chat_full, (uint32_t)kTileRows * p.k * 4u);
@@ -1032,8 +1035,8 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                     __syncwarp();
                     if (lane == 0) {
                         if (slab_live)
-                            tma_store_3d(&tm_rout, stage0 + s * kTileBytes + (uint32_t)q * kSlabBytes, c * kTileCols,
-                                         slab_row0, un.b);
+                            tma_store_3d_hint(&tm_rout, stage0 + s * kTileBytes + (uint32_t)q * kSlabBytes, c * kTileCols,
+                                              slab_row0, un.b, pol_store);
                         tma_store_commit();
                         // the slot goes back once its store has read it: checked one chunk late, so
                         // the warp does not sit out the store it has just issued
