@@ -1739,8 +1739,16 @@ bool fill_full(const StepArgs &a, UmmaParams &p, int cluster = 1) {
     if (!fill_params(a, p)) return false;
     p.cluster = cluster;
     fill_groups(a, p);
+    const bool a_tmem = a.k >= 64 && cluster == 1;
+    // With the operand in TMEM the basis slices may outgrow the 32 KB of fill_groups: wider groups
+    // mean fewer, wider MMAs in pass 2 (N = 192 costs ~144 cycles, two of N = 128 ~230) and fewer
+    // hand-overs per unit -- as wide as TMEM and, below, shared memory allow (measured: k = 128
+    // +4 %, k = 256 +44 % over slices of 32 KB).
+    if (a_tmem) p.gc = 4;
     // TMEM: C in columns [0, k), then the pass-2 ring; at least two ring stages
     while (p.gc > 1 && a.k + 2 * p.gc * kTileCols > 512) --p.gc;
+    // shared memory: two basis slices and at least six F slots
+    while (a_tmem && p.gc > 1 && 2 * (size_t)p.gc * kTileCols * a.k * 2 + 6 * (size_t)kTileBytes > kSmemBudget - 2048 - kBarBytes) --p.gc;
     p.acc_cols = p.gc * kTileCols;
     p.acc_stages = (512 - a.k) / p.acc_cols < kAccStages ? (512 - a.k) / p.acc_cols : kAccStages;
     p.vslice_bytes = (uint32_t)p.gc * kTileCols * a.k * 2;
@@ -1749,7 +1757,6 @@ bool fill_full(const StepArgs &a, UmmaParams &p, int cluster = 1) {
     // a third basis slot first (a slice arrives 2000-3000 cycles after its request under load, a
     // group of MMAs lasts ~1000), a fourth if it costs no F slot.  Below k = 64, and in a cluster,
     // the operand and the staged Chat share a region of shared memory.
-    const bool a_tmem = a.k >= 64 && cluster == 1;
     p.chat_stage_off = a_tmem ? 0u : p.a_bytes;
     p.a_region_bytes = a_tmem ? 0u : p.a_bytes + (uint32_t)kTileRows * a.k * 4u;
     p.a_region_bytes = (p.a_region_bytes + 1023u) & ~1023u;
