@@ -103,6 +103,7 @@ SHAPES = [
     (300, 1152, 64, "bf16", 0),
     (257, 3072, 128, "bf16", 0),
     (1000, 512, 256, "bf16", 0),
+    (200, 768, 192, "bf16", 0),     # three K blocks: operand in tensor memory, previous Chat fetched per block
     (515, 1024, 16, "bf16", 0),
     (384, 2048, 32, "bf16", 64),
     (40, 8192, 64, "bf16", 0),
