@@ -40,7 +40,7 @@ int ritz_width(int D, int k) {
 }
 
 struct CalibLayout {
-    size_t G, gram_scratch, Q, Z, T, S, W, X, theta, resid, scal, dead, total;
+    size_t G, gram_scratch, Q, Z, T, S, W, X, theta, resid, scal, dead, partials, partial_bytes, total;
     int m;
 };
 
@@ -61,9 +61,14 @@ CalibLayout calib_layout(int D, int k) {
     L.resid = at; at += align_up((size_t)L.m * 8, kAlign);
     L.scal = at; at += kAlign;
     L.dead = at; at += align_up((size_t)L.m * 4, kAlign);
+    // partial products of the solver's split GEMMs (see dgemm); small problems do without
+    L.partial_bytes = D >= 1024 ? align_up(std::max((size_t)8 * D * L.m, (size_t)96 * L.m * L.m) * 8, kAlign) : 0;
+    L.partials = at; at += L.partial_bytes;
     L.total = at;
     return L;
 }
+
+int grid_for(int64_t n) { return (int)std::min<int64_t>((n + 255) / 256, 148 * 8); }
 
 template <typename T> __device__ __forceinline__ double to_double(T x);
 template <> __device__ __forceinline__ double to_double<double>(double x) { return x; }
@@ -78,13 +83,17 @@ template <> __device__ __forceinline__ double to_double<__nv_bfloat16>(__nv_bflo
 //   A_T = false:  A(l, i) = A[i * lda + l]     ("NN")
 // 64 x 64 tile of C per CTA, 4 x 4 outputs per thread, 16-deep shared-memory slabs.
 // upper_only: only tiles with tj >= ti are computed (C symmetric, mirrored later).
+// The solver's products are tall and skinny (G Q: 48 x 2 tiles; Q^T Z: 2 x 2 tiles, each with
+// a reduction 3072 long), far too few CTAs for 148 SMs: with ksplit > 1, blockIdx.y takes a
+// slice of the reduction and writes its partial tile to P[y][Md][Nd]; sum_partials_kernel
+// adds the slices in order (no atomics: the result does not depend on timing).
 // ---------------------------------------------------------------------------------------
 constexpr int GT = 64, GK = 16;
 
 template <typename TA, typename TB, bool A_T>
 __global__ void __launch_bounds__(256)
 dgemm_kernel(const TA *__restrict__ A, int64_t lda, const TB *__restrict__ B, int64_t ldb, double *C,
-             int64_t ldc, int Md, int Nd, int64_t L, int accumulate, int upper_only) {
+             int64_t ldc, int Md, int Nd, int64_t L, int accumulate, int upper_only, int ksplit, double *P) {
     __shared__ double As[GK][GT + 2];
     __shared__ double Bs[GK][GT + 2];
     int ti, tj;
@@ -107,7 +116,10 @@ dgemm_kernel(const TA *__restrict__ A, int64_t lda, const TB *__restrict__ B, in
 #pragma unroll
         for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
 
-    for (int64_t l0 = 0; l0 < L; l0 += GK) {
+    const int64_t Lc = ksplit > 1 ? ((L + (int64_t)ksplit * GK - 1) / ((int64_t)ksplit * GK)) * GK : L;
+    const int64_t l_begin = (int64_t)blockIdx.y * Lc;
+    L = l_begin + Lc < L ? l_begin + Lc : L;   // this CTA's slice of the reduction
+    for (int64_t l0 = l_begin; l0 < L; l0 += GK) {
         for (int e = threadIdx.x; e < GK * GT; e += 256) {
             int kk, ii;
             if (A_T) { kk = e / GT; ii = e % GT; } else { ii = e / GK; kk = e % GK; }
@@ -144,20 +156,46 @@ dgemm_kernel(const TA *__restrict__ A, int64_t lda, const TB *__restrict__ B, in
         for (int v = 0; v < 4; ++v) {
             const int j = j0 + tx * 4 + v;
             if (j >= Nd) continue;
-            double *c = C + (int64_t)i * ldc + j;
-            *c = accumulate ? (*c + acc[u][v]) : acc[u][v];
+            if (ksplit > 1) {
+                P[((int64_t)blockIdx.y * Md + i) * Nd + j] = acc[u][v];
+            } else {
+                double *c = C + (int64_t)i * ldc + j;
+                *c = accumulate ? (*c + acc[u][v]) : acc[u][v];
+            }
         }
     }
 }
 
+__global__ void sum_partials_kernel(const double *P, int ksplit, double *C, int64_t ldc, int Md, int Nd, int accumulate) {
+    const int64_t n = (int64_t)Md * Nd;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x) {
+        double acc = 0.0;
+        for (int y = 0; y < ksplit; ++y) acc += P[(int64_t)y * n + e];
+        double *c = C + (e / Nd) * ldc + (e % Nd);
+        *c = accumulate ? (*c + acc) : acc;
+    }
+}
+
+// scratch for split reductions (may be empty: then every product is one CTA deep)
+struct Partials { double *buf = nullptr; size_t bytes = 0; };
+
 template <typename TA, typename TB, bool A_T>
 int dgemm(const TA *A, int64_t lda, const TB *B, int64_t ldb, double *C, int64_t ldc, int Md, int Nd,
-          int64_t L, bool accumulate, bool upper_only, cudaStream_t s) {
+          int64_t L, bool accumulate, bool upper_only, cudaStream_t s, Partials ps = Partials()) {
     const int nti = (Md + GT - 1) / GT, ntj = (Nd + GT - 1) / GT;
     const int blocks = upper_only ? nti * (nti + 1) / 2 : nti * ntj;
-    dgemm_kernel<TA, TB, A_T><<<blocks, 256, 0, s>>>(A, lda, B, ldb, C, ldc, Md, Nd, L, accumulate ? 1 : 0,
-                                                     upper_only ? 1 : 0);
+    // enough CTAs for ~4 per SM, slices at least two slabs deep, and what the scratch holds
+    int64_t ks = upper_only ? 1 : (4 * 148 + blocks - 1) / blocks;
+    ks = std::min<int64_t>(ks, L / (2 * GK));
+    ks = std::min<int64_t>(ks, (int64_t)(ps.bytes / ((size_t)Md * Nd * 8)));
+    if (ks < 2 || ps.buf == nullptr) ks = 1;
+    dgemm_kernel<TA, TB, A_T><<<dim3(blocks, (unsigned)ks), 256, 0, s>>>(A, lda, B, ldb, C, ldc, Md, Nd, L, accumulate ? 1 : 0,
+                                                                        upper_only ? 1 : 0, (int)ks, ps.buf);
     count_launch();
+    if (ks > 1) {
+        sum_partials_kernel<<<grid_for((int64_t)Md * Nd), 256, 0, s>>>(ps.buf, (int)ks, C, ldc, Md, Nd, accumulate ? 1 : 0);
+        count_launch();
+    }
     return check_last_launch();
 }
 
@@ -305,9 +343,19 @@ __global__ void reseed_dead_kernel(double *Q, int D, int m, const int *dead, uin
 // (m/2)^2 blocks update independently.  m must be even.
 // ---------------------------------------------------------------------------------------
 constexpr int kMaxRitz = 384;
+constexpr size_t kJacobiSmemMax = 200 * 1024;   // S and W of the Ritz problem in shared memory when they fit (m <= 113)
 
 __global__ void __launch_bounds__(1024)
-jacobi_kernel(double *S, double *W, double *Wout, double *theta, int m, double *sweeps_out) {
+jacobi_kernel(double *S_g, double *W_g, double *Wout, double *theta, int m, double *sweeps_out, int in_smem) {
+    // A round is a handful of dependent accesses between barriers: with S and W in global memory
+    // each costs an L2 round trip (~1.4 ms per call at m = 80); when both fit they live in shared
+    // memory for the whole call.
+    extern __shared__ double jacobi_dyn[];
+    double *S = in_smem ? jacobi_dyn : S_g;
+    double *W = in_smem ? jacobi_dyn + (size_t)m * m : W_g;
+    if (in_smem) {
+        for (int e = threadIdx.x; e < m * m; e += blockDim.x) S[e] = S_g[e];
+    }
     __shared__ double cs_c[kMaxRitz / 2], cs_s[kMaxRitz / 2];
     __shared__ int pr_p[kMaxRitz / 2], pr_q[kMaxRitz / 2];
     __shared__ int s_rot;
@@ -446,7 +494,6 @@ __global__ void emit_basis_kernel(const double *Q, const double *theta, int D, i
 
 __global__ void copy_scalar_kernel(const double *src, double *dst) { *dst = *src; }
 
-int grid_for(int64_t n) { return (int)std::min<int64_t>((n + 255) / 256, 148 * 8); }
 
 }  // namespace
 
@@ -489,10 +536,10 @@ namespace {
 // found dependent in the first pass are re-seeded before the second).  Zin is destroyed;
 // T is scratch.  The result ends up in Zin's buffer, returned through *out.
 int orthonormalize(double *Zin, double *T, double *S, double *X, int *dead, int D, int m, uint64_t salt,
-                   double **out, cudaStream_t s) {
+                   double **out, cudaStream_t s, Partials ps) {
     double *src = Zin, *dst = T;
     for (int pass = 0; pass < 2; ++pass) {
-        int rc = dgemm<double, double, true>(src, m, src, m, S, m, m, m, D, false, false, s);
+        int rc = dgemm<double, double, true>(src, m, src, m, S, m, m, m, D, false, false, s, ps);
         if (rc) return rc;
         symmetrize_kernel<<<grid_for((int64_t)m * m), 256, 0, s>>>(S, m, 1);
         chol_inv_kernel<<<1, 1024, 0, s>>>(S, X, m, dead);
@@ -542,7 +589,8 @@ int calib_finish(int D, int k, float *Vk, double *lambda, double *trace, double 
 
     int *dead = (int *)(w + L.dead);
     double *Q = nullptr;
-    rc = orthonormalize(bufA, bufB, S, X, dead, D, m, 1, &Q, s);
+    const Partials ps{(double *)(w + L.partials), L.partial_bytes};
+    rc = orthonormalize(bufA, bufB, S, X, dead, D, m, 1, &Q, s, ps);
     if (rc) return rc;
     auto others = [&](double *q, double **z, double **t) {
         double *all[3] = {bufA, bufB, bufC};
@@ -564,13 +612,21 @@ int calib_finish(int D, int k, float *Vk, double *lambda, double *trace, double 
     while (mult < max_mult) {
         double *Z, *T;
         others(Q, &Z, &T);
-        rc = dgemm<double, double, true>(G, D, Q, m, Z, m, D, m, D, false, false, s);   // Z = G Q
+        rc = dgemm<double, double, true>(G, D, Q, m, Z, m, D, m, D, false, false, s, ps);   // Z = G Q
         if (rc) return rc;
         ++mult;
-        rc = dgemm<double, double, true>(Q, m, Z, m, S, m, m, m, D, false, false, s);   // S = Q^T Z
+        rc = dgemm<double, double, true>(Q, m, Z, m, S, m, m, m, D, false, false, s, ps);   // S = Q^T Z
         if (rc) return rc;
         symmetrize_kernel<<<grid_for((int64_t)m * m), 256, 0, s>>>(S, m, 1);
-        jacobi_kernel<<<1, 1024, 0, s>>>(S, X, W, theta, m, scal + 2);
+        {
+            const size_t jb = 2 * (size_t)m * m * 8;
+            const bool fits = jb <= kJacobiSmemMax;
+            if (fits && jb > 40 * 1024) {   // per call: the attribute belongs to the current device's copy of the kernel
+                rc = record_cuda(cudaFuncSetAttribute(jacobi_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kJacobiSmemMax));
+                if (rc) return rc;
+            }
+            jacobi_kernel<<<1, 1024, fits ? jb : 0, s>>>(S, X, W, theta, m, scal + 2, fits ? 1 : 0);
+        }
         count_launch(2);
         rc = dgemm<double, double, false>(Q, m, W, m, T, m, D, m, m, false, false, s);  // ritz = Q W
         if (rc) return rc;
@@ -592,7 +648,7 @@ int calib_finish(int D, int k, float *Vk, double *lambda, double *trace, double 
                 break;
             }
         }
-        rc = orthonormalize(image, Z, S, X, dead, D, m, (uint64_t)mult + 1, &Q, s);
+        rc = orthonormalize(image, Z, S, X, dead, D, m, (uint64_t)mult + 1, &Q, s, ps);
         if (rc) return rc;
     }
 
