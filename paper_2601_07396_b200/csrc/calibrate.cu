@@ -343,6 +343,7 @@ __global__ void reseed_dead_kernel(double *Q, int D, int m, const int *dead, uin
 // (m/2)^2 blocks update independently.  m must be even.
 // ---------------------------------------------------------------------------------------
 constexpr int kMaxRitz = 384;
+constexpr int kJacobiThreads = 1024;
 constexpr size_t kJacobiSmemMax = 200 * 1024;   // S and W of the Ritz problem in shared memory when they fit (m <= 113)
 
 __global__ void __launch_bounds__(1024)
@@ -378,12 +379,15 @@ jacobi_kernel(double *S_g, double *W_g, double *Wout, double *theta, int m, doub
                 pr_p[tid] = p; pr_q[tid] = q;
                 const double app = S[(int64_t)p * m + p], aqq = S[(int64_t)q * m + q], apq = S[(int64_t)p * m + q];
                 double c = 1.0, s = 0.0;
-                if (apq != 0.0 && fabs(apq) > 1e-17 * sqrt(fabs(app * aqq)) ) {
+                // (thresholds on squares: this chain of fp64 divisions and roots is the serial part of
+                // every round, so it does without the square root of |app aqq|)
+                const double pq2 = apq * apq, dd = fabs(app * aqq);
+                if (apq != 0.0 && pq2 > 1e-34 * dd) {
                     const double tau = (aqq - app) / (2.0 * apq);
                     const double t = (tau >= 0.0 ? 1.0 : -1.0) / (fabs(tau) + sqrt(1.0 + tau * tau));
-                    c = 1.0 / sqrt(1.0 + t * t);
+                    c = rsqrt(1.0 + t * t);
                     s = t * c;
-                    if (fabs(apq) > 1e-15 * sqrt(fabs(app * aqq))) atomicAdd(&s_rot, 1);
+                    if (pq2 > 1e-30 * dd) atomicAdd(&s_rot, 1);
                 }
                 cs_c[tid] = c; cs_s[tid] = s;
             }
@@ -625,7 +629,7 @@ int calib_finish(int D, int k, float *Vk, double *lambda, double *trace, double 
                 rc = record_cuda(cudaFuncSetAttribute(jacobi_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kJacobiSmemMax));
                 if (rc) return rc;
             }
-            jacobi_kernel<<<1, 1024, fits ? jb : 0, s>>>(S, X, W, theta, m, scal + 2, fits ? 1 : 0);
+            jacobi_kernel<<<1, kJacobiThreads, fits ? jb : 0, s>>>(S, X, W, theta, m, scal + 2, fits ? 1 : 0);
         }
         count_launch(2);
         rc = dgemm<double, double, false>(Q, m, W, m, T, m, D, m, m, false, false, s);  // ritz = Q W
