@@ -177,7 +177,8 @@ __device__ __forceinline__ int last_own_chunk(uint32_t it0, int nsub, uint32_t g
 // tiles of the group's chunks stream through their own ring and meet the accumulator in
 // the epilogue.
 //
-// Warp roles (320 threads): 0 = TMA producer, 1 = MMA issuer (+ TMEM owner), 2..9 = two
+// Warp roles (320 threads): 0 = TMA producer (lane 0: R tiles and basis slices, lane 1: A tiles),
+// 1 = MMA issuer (+ TMEM owner), 2..9 = two
 // epilogue groups of four warps (TMEM lane quarter = warp % 4; group g takes the chunks
 // whose running index is g modulo 2).  Each epilogue warp owns a 32-row slab of the chunk
 // from the TMEM read to its own TMA store, so the eight warps never meet at a barrier.
@@ -230,36 +231,39 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer ---
+        // The A tile of live unit number ua (of unit ux): with two operand buffers (k <= 64) the
+        // requests run on a lane of their own, one unit ahead of the MMAs, and never hold up the R
+        // and basis streams (+4 % on the FLUX shape); with a single buffer the tile can only be
+        // requested when the MMAs of the unit before are done, and it goes first, in order, on the
+        // stream lane -- R tiles requested ahead of it only delay it (measured at k = 128).
+        auto request_a = [&](const Unit &ux, uint32_t ua) {
+            const uint32_t ab = ua % p.a_bufs;
+            SVDC_TRACE_MARK(p0);
+            if (!mbar_wait(bar.a_empty + 8 * ab, ((ua / p.a_bufs) & 1u) ^ 1u, abort_flag, 1)) return false;
+            SVDC_TRACE_ADD(0, p0);
+            const uint32_t dst = a_base0 + ab * p.a_bytes;
+            mbar_arrive_expect_tx(bar.a_full + 8 * ab, p.a_bytes);
+            for (int kb = 0; kb < p.nkb; ++kb) {
+                tma_load_3d(dst + kb * (kTileRows * p.kb_bytes), &tm_ahi, bar.a_full + 8 * ab,
+                            kb * p.kb_elems, ux.rt * kTileRows, ux.b);
+                tma_load_3d(dst + p.a_half_bytes + kb * (kTileRows * p.kb_bytes), &tm_alo, bar.a_full + 8 * ab,
+                            kb * p.kb_elems, ux.rt * kTileRows, ux.b);
+            }
+            return true;
+        };
         if (lane == 0) {
-            uint32_t ui = 0, ua = 0;                   // units started; A tiles requested
             RingPos fr, vr;                            // next R slot, next basis slot
-            int u_a = blockIdx.x;                      // unit cursor of the A-tile requests (runs ahead)
+            uint32_t ua = 0;
             for (int u = blockIdx.x; u < p.units; u += gridDim.x) {
                 const Unit un = decode_unit(p, u);
                 if (*(volatile uint32_t *)&header_of(p, un.b)->full_steps == 0) {
                     if (un.rt == 0 && un.c0 == 0) header_of(p, un.b)->status = SVDCACHE_ERR_STATE;
                     continue;
                 }
-                // request the A tiles of this unit and of the next a_bufs - 1 live units
-                while (ua < ui + (uint32_t)p.a_bufs && u_a < p.units) {
-                    const Unit ux = decode_unit(p, u_a);
-                    u_a += gridDim.x;
-                    if (*(volatile uint32_t *)&header_of(p, ux.b)->full_steps == 0) continue;
-                    const uint32_t ab = ua % p.a_bufs;
-                    SVDC_TRACE_MARK(p0);
-                    if (!mbar_wait(bar.a_empty + 8 * ab, ((ua / p.a_bufs) & 1u) ^ 1u, abort_flag, 1)) { record_timeout(p, abort_flag); goto done; }
-                    SVDC_TRACE_ADD(0, p0);
-                    const uint32_t dst = a_base0 + ab * p.a_bytes;
-                    mbar_arrive_expect_tx(bar.a_full + 8 * ab, p.a_bytes);
-                    for (int kb = 0; kb < p.nkb; ++kb) {
-                        tma_load_3d(dst + kb * (kTileRows * p.kb_bytes), &tm_ahi, bar.a_full + 8 * ab,
-                                    kb * p.kb_elems, ux.rt * kTileRows, ux.b);
-                        tma_load_3d(dst + p.a_half_bytes + kb * (kTileRows * p.kb_bytes), &tm_alo, bar.a_full + 8 * ab,
-                                    kb * p.kb_elems, ux.rt * kTileRows, ux.b);
-                    }
+                if (p.a_bufs == 1) {
+                    if (!request_a(un, ua)) { record_timeout(p, abort_flag); goto done; }
                     ++ua;
                 }
-                ++ui;
                 for (int cg = un.c0; cg < un.c1; cg += p.gc) {
                     const uint32_t vs = vr.idx;
                     SVDC_TRACE_MARK(p1);
@@ -282,6 +286,14 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
                         tma_load_3d(stage0 + s * kTileBytes, &tm_r, bar.full + 8 * s, c * kTileCols, un.rt * kTileRows, un.b);
                     }
                 }
+            }
+        } else if (lane == 1 && p.a_bufs > 1) {
+            uint32_t ua = 0;
+            for (int u = blockIdx.x; u < p.units; u += gridDim.x) {
+                const Unit ux = decode_unit(p, u);
+                if (*(volatile uint32_t *)&header_of(p, ux.b)->full_steps == 0) continue;
+                if (!request_a(ux, ua)) { record_timeout(p, abort_flag); goto done; }
+                ++ua;
             }
         }
     } else if (warp == 1) {
