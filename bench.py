@@ -40,7 +40,7 @@ NOMINAL_HBM_GBS = 8000.0
 # profiles/umma_cached_kernel_flux_8blocks.txt: taken on 8 blocks of the same shape and
 # scaled by the block count (traffic is proportional to the blocks a launch covers).  The
 # tail of the output that is still in L2 when the kernel ends is not in the counter.
-NCU_TRAFFIC_BYTES_PER_BLOCK = {("flux", 2): 51901088}
+NCU_TRAFFIC_BYTES_PER_BLOCK = {("flux", 2): 52100928}
 
 
 def algorithmic_bytes(spec: streams.StreamSpec, nblocks: int):
