@@ -1881,19 +1881,37 @@ bool umma_supported(const StepArgs &a, bool full) {
 int umma_cached_step(const StepArgs &a, cudaStream_t s) {
     UmmaParams p{};
     if (!fill_cached(a, p)) return SVDCACHE_ERR_BAD_SHAPE;
-    // Split D across CTAs only when there are too few row tiles to occupy the GPU: pick the
-    // split (in whole MMA groups) that minimises the chunks the busiest CTA has to stream.
+    // Units: a row tile, or a column range of it (in whole MMA groups).  The split is the one that
+    // minimises what the busiest CTA has to stream, in chunks of R + Fhat traffic (32 KB) -- and,
+    // among splits within 2 % of that, the finest when the operand is double-buffered: CTAs that
+    // work on neighbouring column ranges of the same rows at the same time read and write whole
+    // DRAM pages together (measured on the FLUX shape: 6.3 TB/s with single-group units, 5.7 with
+    // whole tiles).  With a single operand buffer (k >= 128) every unit waits for its own copy of
+    // the tile's A operand with empty rings (~4 chunks' worth, plus the a_bytes it re-reads), which
+    // outweighs that: 5.7 TB/s with whole tiles at k = 128, 4.2 with single-group units.
     const int tiles = p.row_tiles * a.nblocks;
     const int groups_total = (p.chunks_total + p.gc - 1) / p.gc;
+    const int unit_cost = p.a_bufs == 1 ? (int)((p.a_bytes + 2 * kTileBytes - 1) / (2 * kTileBytes)) + 4 : 0;
+    auto load_of = [&](int ds, int *eff_out, int *gps_out) {
+        const int gps = (groups_total + ds - 1) / ds;            // groups per slice
+        const int eff = (groups_total + gps - 1) / gps;          // slices that result
+        const int rounds = (tiles * eff + num_sms() - 1) / num_sms();
+        *eff_out = eff; *gps_out = gps;
+        return rounds * (gps * p.gc + unit_cost);
+    };
     int best_load = 1 << 30;
     p.dsplit = 1;
     p.chunks_per_slice = p.chunks_total;
     for (int ds = 1; ds <= groups_total && ds <= 16; ++ds) {
-        const int gps = (groups_total + ds - 1) / ds;            // groups per slice
-        const int eff = (groups_total + gps - 1) / gps;          // slices that result
-        const int rounds = (tiles * eff + num_sms() - 1) / num_sms();
-        if (rounds * gps < best_load) { best_load = rounds * gps; p.dsplit = eff; p.chunks_per_slice = gps * p.gc; }
+        int eff, gps;
+        const int load = load_of(ds, &eff, &gps);
+        if (load < best_load) { best_load = load; p.dsplit = eff; p.chunks_per_slice = gps * p.gc; }
     }
+    if (p.a_bufs > 1)
+        for (int ds = 1; ds <= groups_total && ds <= 16; ++ds) {
+            int eff, gps;
+            if (load_of(ds, &eff, &gps) * 50 <= best_load * 51 && eff > p.dsplit) { p.dsplit = eff; p.chunks_per_slice = gps * p.gc; }
+        }
     p.units = tiles * p.dsplit;
 
     const StateLayout SL = state_layout(a.N, a.D, a.k, a.dtype);
