@@ -231,21 +231,26 @@ SVDCACHE_API int svdcache_cached_step_batched(int nblocks, const void *state, si
 /* ---------------------------------------------------------------------------------
  * Introspection for benchmarks and tests (host only).
  *   svdcache_kernel_launches: kernels this library has launched in this process.
- *   svdcache_set_path: 0 = pick automatically, 1 = force the CUDA-core kernels,
- *                      2 = force the tcgen05 kernels (error if the shape is outside
- *                      what they support), 3 = as 2, and the full step shares each
- *                      128-row tile between the two CTAs of a thread-block cluster
- *                      (each streams half of the columns; the partial coefficients
- *                      meet through distributed shared memory) where the shape
- *                      allows it, 4 = as 2, with the experimental batched two-phase full
- *                      step (every tile's columns shared by up to eight CTAs, partial
- *                      coefficients combined through memory, pass 2 one or two batches
- *                      after pass 1).  Returns the previous setting.
- *   svdcache_last_path: which kernel family the last step call used (1 .. 4).
+ *   svdcache_set_path: a process-wide switch for tests and benchmarks (every later step call
+ *                      of every thread sees it; not meant for production code).
+ *                      0 = pick automatically, 1 = force the CUDA-core kernels,
+ *                      2 = force the tcgen05 kernels (error if the shape is outside what
+ *                      they support).  Returns the previous setting.
+ *   svdcache_last_path: which kernel family the last step call used (1 or 2).
  * ------------------------------------------------------------------------------- */
 SVDCACHE_API uint64_t svdcache_kernel_launches(void);
 SVDCACHE_API int svdcache_set_path(int path);
 SVDCACHE_API int svdcache_last_path(void);
+
+/* Self-test of the time-out path (no counterpart in the paper).  Every wait inside the
+ * tcgen05 kernels is bounded (~2 s): when one runs out the kernel stops, stores
+ * SVDCACHE_ERR_TIMEOUT in the state header of block 0 together with which wait it was, and
+ * returns, so the context stays usable.  This call launches one small CTA that waits, with the
+ * same code, for an event that never comes, for `limit_cycles` SM cycles (1 .. 2e8): afterwards
+ * svdcache_state_query on `state` (a reset state buffer, device, 256-byte aligned) must report
+ * SVDCACHE_ERR_TIMEOUT, the word at byte 36 of the header reads 99 << 16 (wait site 99, CTA 0),
+ * and svdcache_state_reset clears both.  Asynchronous on `stream`.  Nothing is faulted or hung. */
+SVDCACHE_API int svdcache_selftest_wait_timeout(void *state, int64_t limit_cycles, void *stream);
 
 #ifdef __cplusplus
 }

@@ -50,6 +50,7 @@ SIGNATURES = {
     "svdcache_kernel_launches": (ctypes.c_uint64, []),
     "svdcache_set_path": (_ci, [_ci]),
     "svdcache_last_path": (_ci, []),
+    "svdcache_selftest_wait_timeout": (_ci, [_vp, _i64, _vp]),
 }
 
 
@@ -289,6 +290,10 @@ def svdcache_set_path(path: int) -> int:
 
 def svdcache_last_path() -> int:
     return int(lib().svdcache_last_path())
+
+
+def svdcache_selftest_wait_timeout(state: torch.Tensor, limit_cycles: int, stream=None) -> None:
+    _check(lib().svdcache_selftest_wait_timeout(_ptr(state), int(limit_cycles), _stream(stream)), "selftest_wait_timeout")
 
 
 # ---------------------------------------------------------- views for tests/tools ---

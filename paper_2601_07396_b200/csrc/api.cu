@@ -41,16 +41,14 @@ static int dispatch(const StepArgs &a_in, bool full, cudaStream_t s) {
     StepArgs a = a_in;
     const int want = g_path.load();
     const bool can_umma = umma_supported(a, full);
-    if (want >= 2 && !can_umma) return SVDCACHE_ERR_BAD_SHAPE;
-    const bool use_umma = (want >= 2) || (want == 0 && can_umma);
-    a.cluster_split = (want == 3) ? 1 : (want == 4) ? 2 : 0;
-    g_last_path.store(use_umma ? (want >= 3 ? want : 2) : 1);
+    if (want == 2 && !can_umma) return SVDCACHE_ERR_BAD_SHAPE;
+    const bool use_umma = (want == 2) || (want == 0 && can_umma);
+    g_last_path.store(use_umma ? 2 : 1);
     if (use_umma) return full ? umma_full_step(a, s) : umma_cached_step(a, s);
     return full ? simt_full_step(a, s) : simt_cached_step(a, s);
 }
 
-__global__ void state_reset_kernel(StateHeader *h, int64_t N, int D, int k, int dtype, uint32_t *sync, int sync_words) {
-    for (int i = threadIdx.x; i < sync_words; i += blockDim.x) sync[i] = 0u;   // per-tile counters and ready marks
+__global__ void state_reset_kernel(StateHeader *h, int64_t N, int D, int k, int dtype) {
     if (threadIdx.x == 0 && blockIdx.x == 0) {
         h->magic = kStateMagic;
         h->dtype = dtype;
@@ -61,6 +59,7 @@ __global__ void state_reset_kernel(StateHeader *h, int64_t N, int D, int k, int 
         h->status = SVDCACHE_OK;
         h->done = 0;
         h->pad = 0;
+        h->exits = 0;
     }
 }
 
@@ -90,10 +89,17 @@ const char *svdcache_last_cuda_error(void) { return g_cuda_error; }
 
 uint64_t svdcache_kernel_launches(void) { return g_launches.load(); }
 int svdcache_set_path(int path) {
-    if (path < 0 || path > 4) return SVDCACHE_ERR_INVALID_ARG;
+    if (path < 0 || path > 2) return SVDCACHE_ERR_INVALID_ARG;
     return g_path.exchange(path);
 }
 int svdcache_last_path(void) { return g_last_path.load(); }
+
+int svdcache_selftest_wait_timeout(void *state, int64_t limit_cycles, void *stream) {
+    if (!state) return SVDCACHE_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(state) & 255u) != 0) return SVDCACHE_ERR_BAD_ALIGN;
+    if (limit_cycles < 1 || limit_cycles > 200000000LL) return SVDCACHE_ERR_INVALID_ARG;   // at most ~0.1 s
+    return umma_wait_selftest(state, (long long)limit_cycles, (cudaStream_t)stream);
+}
 
 /* ----------------------------------------------------------------- calibration --- */
 
@@ -221,10 +227,7 @@ int svdcache_state_reset(void *state, int64_t N, int D, int k, int dtype, void *
     if (rc) return rc;
     if (!state) return SVDCACHE_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(state) & 255u) != 0) return SVDCACHE_ERR_BAD_ALIGN;
-    const StateLayout SL = state_layout(N, D, k, dtype);
-    state_reset_kernel<<<1, 256, 0, (cudaStream_t)stream>>>((StateHeader *)state, N, D, k, dtype,
-                                                            reinterpret_cast<uint32_t *>((char *)state + SL.sync),
-                                                            (int)((SL.r - SL.sync) / 4));
+    state_reset_kernel<<<1, 32, 0, (cudaStream_t)stream>>>((StateHeader *)state, N, D, k, dtype);
     count_launch();
     return check_last_launch();
 }

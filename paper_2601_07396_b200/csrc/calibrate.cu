@@ -208,7 +208,12 @@ __global__ void init_header_kernel(CalibHeader *h, int D, int k) {
     h->D = D; h->k_max = k; h->rows = 0; h->status = SVDCACHE_OK;
 }
 
-__global__ void add_rows_kernel(CalibHeader *h, int64_t M) { h->rows += M; }
+// counts the rows of a chunk; a chunk of another width than the accumulation was begun with
+// poisons the header, so that the finish refuses it
+__global__ void add_rows_kernel(CalibHeader *h, int64_t M, int D) {
+    h->rows += M;
+    if (h->D != D && h->status == SVDCACHE_OK) h->status = SVDCACHE_ERR_WORKSPACE;
+}
 
 // lower <- upper (mode 0), or S <- (S + S^T)/2 (mode 1)
 __global__ void symmetrize_kernel(double *A, int n, int mode) {
@@ -529,7 +534,7 @@ int calib_accumulate(const void *F, int64_t M, int D, int64_t ld, int dtype, voi
         rc = dgemm<float, float, true>(f, ld, f, ld, G, D, D, D, M, true, true, s);
     }
     if (rc) return rc;
-    add_rows_kernel<<<1, 1, 0, s>>>((CalibHeader *)w, M);
+    add_rows_kernel<<<1, 1, 0, s>>>((CalibHeader *)w, M, D);
     count_launch();
     return check_last_launch();
 }
@@ -574,13 +579,7 @@ int calib_finish(int D, int k, float *Vk, double *lambda, double *trace, double 
     double *theta = (double *)(w + L.theta), *resid = (double *)(w + L.resid), *scal = (double *)(w + L.scal);
     // scal[0] = trace, scal[1] = max relative residual, scal[2] = Jacobi sweeps
 
-    symmetrize_kernel<<<grid_for((int64_t)D * D), 256, 0, s>>>(G, D, 0);
-    trace_kernel<<<1, 256, 0, s>>>(G, D, scal);
-    init_block_kernel<<<grid_for((int64_t)D * m), 256, 0, s>>>(bufA, (int64_t)D * m);
-    count_launch(3);
-    int rc = check_last_launch();
-    if (rc) return rc;
-
+    int rc;
     // an accumulation kernel whose bounded wait ran out has left its error in the header
     {
         CalibHeader h;
@@ -589,7 +588,18 @@ int calib_finish(int D, int k, float *Vk, double *lambda, double *trace, double 
         rc = record_cuda(cudaStreamSynchronize(s));
         if (rc) return rc;
         if (h.status != SVDCACHE_OK) return h.status;
+        // the workspace must be the one svdcache_calibrate_begin laid out for this width, and for a
+        // rank at least as large (G sits at a fixed offset; the solver's buffers grow with k)
+        if (h.D != D || k > h.k_max) return SVDCACHE_ERR_WORKSPACE;
     }
+
+    symmetrize_kernel<<<grid_for((int64_t)D * D), 256, 0, s>>>(G, D, 0);
+    trace_kernel<<<1, 256, 0, s>>>(G, D, scal);
+    init_block_kernel<<<grid_for((int64_t)D * m), 256, 0, s>>>(bufA, (int64_t)D * m);
+    count_launch(3);
+    rc = check_last_launch();
+    if (rc) return rc;
+
 
     int *dead = (int *)(w + L.dead);
     double *Q = nullptr;

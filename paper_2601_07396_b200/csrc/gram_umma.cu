@@ -325,11 +325,9 @@ int umma_gram_accumulate(const void *F, int64_t M, int D, int64_t ld, double *G,
     p.units = p.whole + surplus * nseg;
     p.partials = scratch;
     const size_t smem = 1024 + (size_t)kGStages * kGStageBytes + kGBarBytes + 64;
-    static bool attr_set = false;
-    if (!attr_set) {
+    {   // kept per device by the runtime: set on every call
         int rc = record_cuda(cudaFuncSetAttribute(umma_gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         if (rc) return rc;
-        attr_set = true;
     }
     const int grid = p.units < sms ? p.units : sms;
     umma_gram_kernel<<<grid, kGThreads, smem, s>>>(tm, p);

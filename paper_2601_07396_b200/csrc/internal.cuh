@@ -27,8 +27,11 @@ struct StateHeader {   // first 256 bytes of a state buffer
     int32_t D, k;
     uint32_t full_steps;   // full steps seen since the last reset
     int32_t status;        // sticky device status word (SVDCACHE_OK or an error code)
-    uint32_t done;         // CTAs of the running full step that have finished
+    uint32_t done;         // CUDA-core full step: CTAs of this block that have finished
     uint32_t pad;          // which wait ran out first: site << 16 | CTA (diagnosis)
+    // tcgen05 full step, in block 0's header: CTAs of the launch that have left the kernel (the
+    // last one counts the step in every block's header)
+    uint32_t exits;
 };
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -48,27 +51,20 @@ inline BasisLayout basis_layout(int D, int k, int dtype) {
     return L;
 }
 
-// header | Chat fp32 [N x k] | (bf16 only) Chat as a split-bf16 pair: hi [N x k], lo [N x k] |
-// (bf16 only) scratch of the full step: this step's C as a split-bf16 pair, and four words per
-// 128-row tile (two arrival counters, ready mark) | R [N x D].
+// header | Chat fp32 [N x k] | (bf16 only) Chat as a split-bf16 pair: hi [N x k], lo [N x k] | R [N x D].
 // hi = bf16(x), lo = bf16(x - hi).  The pair of Chat is the tensor-core operand of the cached
-// step, written by the full step next to Chat so that the cached step reads it as it is; the
-// pair of C is the operand of the full step's own second pass.
+// step, written by the full step next to Chat so that the cached step reads it as it is.
 struct StateLayout {
-    size_t chat, op_hi, op_lo, c_hi, c_lo, sync, r, total;
+    size_t chat, op_hi, op_lo, r, total;
 };
 inline StateLayout state_layout(int64_t N, int D, int k, int dtype) {
     StateLayout L;
     const bool bf = dtype == SVDCACHE_BF16;
     const size_t op = bf ? align_up((size_t)N * k * 2, kAlign) : 0;
-    const size_t tiles = (size_t)((N + 127) / 128);
     L.chat = kHeaderBytes;
     L.op_hi = L.chat + align_up((size_t)N * k * 4, kAlign);
     L.op_lo = L.op_hi + op;
-    L.c_hi = L.op_lo + op;
-    L.c_lo = L.c_hi + op;
-    L.sync = L.c_lo + op;
-    L.r = L.sync + (bf ? align_up(tiles * 16, kAlign) : 0);
+    L.r = L.op_lo + op;
     L.total = L.r + align_up((size_t)N * D * elem_bytes(dtype), kAlign);
     return L;
 }
@@ -92,8 +88,6 @@ struct StepArgs {
     int64_t N;
     int D, k, dtype, nblocks;
     float beta;
-    int cluster_split;      // full step, tcgen05 family: 1 = share each row tile between the two CTAs of a cluster,
-                            // 2 = batched two-phase schedule (column slices over CTAs, partials through memory)
 };
 
 // launch bookkeeping (api.cu)
@@ -109,6 +103,7 @@ int simt_cached_step(const StepArgs &a, cudaStream_t s);
 bool umma_supported(const StepArgs &a, bool full);
 int umma_full_step(const StepArgs &a, cudaStream_t s);
 int umma_cached_step(const StepArgs &a, cudaStream_t s);
+int umma_wait_selftest(void *state, long long limit_cycles, cudaStream_t s);
 
 // basis (basis.cu)
 int basis_prepare(const float *Vk, int D, int k, int dtype, void *basis, cudaStream_t s);

@@ -44,10 +44,6 @@ struct UmmaParams {
     int dual, acc_stride;                    // cached step: separate hi / lo accumulators; TMEM columns per ring stage
     uint32_t vslice_bytes;
     uint32_t a_region_bytes, chat_stage_off; // full step: A operand (+ Chat staging when it is not in place)
-    int cluster;                             // full step: CTAs that share a row tile (1, or 2 splitting D)
-    // batched two-phase full step: column slices per tile, tiles per batch, batches, tiles in all
-    int Q, Bt, nbat, T, lag;   // lag: pass 2 of a batch runs this many batches after its pass 1
-    size_t chi_off, clo_off, sync_off, r_off;
     char *state;
     size_t state_stride, chat_off, ophi_off, oplo_off;
     float *C_out;
@@ -114,6 +110,24 @@ __device__ __forceinline__ void record_timeout(const UmmaParams &p, volatile int
     if ((*(volatile uint32_t *)&h->pad & 0xFFFFu) == (blockIdx.x & 0xFFFFu) && (threadIdx.x & 31u) == 0u) {
         uint32_t *w = reinterpret_cast<uint32_t *>(h) + 16 + 4 * (threadIdx.x >> 5);
         w[0] = mine; w[1] = c0; w[2] = c1; w[3] = c2;
+    }
+}
+
+// Every CTA of a full-step launch reports here when it has nothing left to do; the last one
+// counts the step in every block's header.  No CTA reads full_steps after its own report, so
+// the first-step test of the EMA (Eq. 11) sees one value for the whole launch, whatever the
+// order in which the warps of a CTA and the CTAs of the grid get to their tiles.
+__device__ __forceinline__ void report_exit_and_count_step(const UmmaParams &p) {
+    StateHeader *h0 = header_of(p, 0);
+    __threadfence();
+    const uint32_t prev = atomicAdd(&h0->exits, 1u);
+    if (prev == gridDim.x - 1u) {
+        __threadfence();
+        for (int b = 0; b < p.nblocks; ++b) {
+            StateHeader *h = header_of(p, b);
+            h->full_steps = h->full_steps + 1;
+        }
+        h0->exits = 0;
     }
 }
 
@@ -458,8 +472,8 @@ done:
 //     split-bf16 copy for the cached step and C_out, and leaves C itself as a split-bf16 A
 //     operand: from k = 64 on in tensor memory, over the columns of C (kTmemA: both epilogue
 //     groups share the job, the previous Chat comes through registers, and all of shared memory
-//     goes to the rings); below that, and in a cluster, in a shared-memory region that also
-//     stages the previous Chat by TMA (warps 6..9 alone).
+//     goes to the rings); below that in a shared-memory region that also stages the previous
+//     Chat by TMA (warps 6..9 alone).
 //   Pass 2 streams the same F chunks again, last group first (the most recently read ones
 //     are the likeliest to sit in L2), with V_k slices of gc*64 rows: C V_k^T per group in
 //     TMEM, and the epilogue stores R = F - C V_k^T through TMA.
@@ -516,7 +530,7 @@ __device__ __forceinline__ void stg256(void *dst, uint4 a, uint4 b) {
                  : "memory");
 }
 
-template <bool kClusterSplit, bool kTmemA>
+template <bool kTmemA>
 __global__ void __launch_bounds__(kThreadsFull, 1)
 umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant__ CUtensorMap tm_vt,
                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_rout,
@@ -531,9 +545,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
     // barriers beyond the ring ones: c_full (C accumulated), a_full (A operand written),
     // p2_done (pass-2 MMAs of the unit finished: the A region may be restaged), chat_full
     // (previous Chat staged)
-    // cluster mode: peer_ready (the peer's A region may be written), recv_full (the peer's
-    // partial C has arrived in mine)
-    const uint32_t chat_full = bar.a_full + 8, p2_done = bar.c_done, peer_ready = bar.a_empty, recv_full = bar.a_empty + 8;
+    const uint32_t chat_full = bar.a_full + 8, p2_done = bar.c_done;
     uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
     volatile int *abort_flag = reinterpret_cast<volatile int *>(gen_base + (bar.abort_flag - base));
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(gen_base + (bar.tmem_slot - base));
@@ -542,22 +554,13 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
     SVDC_TRACE_DECL
     const uint32_t tmem_cols = 512;
     const int CT = p.chunks_total;
-    // A cluster of two CTAs shares each row tile: rank r takes a contiguous range of the
-    // column groups in both passes, the partial C's meet through distributed shared memory.
-    constexpr uint32_t csize = kClusterSplit ? 2u : 1u;
-    const uint32_t crank = kClusterSplit ? cluster_ctarank() : 0u;
-    const int cid = (int)(blockIdx.x / csize), nclusters = (int)(gridDim.x / csize);
-    const int G_all = (CT + p.gc - 1) / p.gc;           // groups per pass, whole width
-    const int g_off = (int)((crank * (uint32_t)G_all) / csize);
-    const int G = (int)(((crank + 1u) * (uint32_t)G_all) / csize) - g_off;   // this CTA's groups per pass
-    const int c_first = g_off * p.gc;
-    const int CTm = min(CT, (g_off + G) * p.gc) - c_first;                   // this CTA's chunks per pass
+    const int cid = (int)blockIdx.x, nctas = (int)gridDim.x;
+    const int G = (CT + p.gc - 1) / p.gc;               // column groups per pass
     const uint32_t a_part = p.k >= 64 ? kBlk32Bytes : p.a_half_bytes;   // hi -> lo distance
-    // From k = 64 on (and without a cluster) the A operand of pass 2 lives in tensor memory, over
-    // C itself, and both epilogue groups share the C job; below that it is staged in shared memory.
+    // From k = 64 on the A operand of pass 2 lives in tensor memory, over C itself, and both
+    // epilogue groups share the C job; below that it is staged in shared memory.
     // (Each variant is an instantiation of its own: compiled together, the two C jobs spill.)
     constexpr bool c_split = kTmemA;
-    static_assert(!(kClusterSplit && kTmemA), "the cluster exchange uses the shared-memory operand region");
     const uint32_t a_kb = 2u * kBlk32Bytes;                             // K-block distance (k >= 64)
 
     if (threadIdx.x == 0) {
@@ -570,8 +573,6 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
         mbar_init(chat_full, 1);
         mbar_init(bar.c_full, 1);
         mbar_init(p2_done, 1);
-        mbar_init(peer_ready, 1);
-        mbar_init(recv_full, 128);
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&tm_f);
@@ -586,7 +587,6 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
     }
     tc_fence_before();
     __syncthreads();
-    if (csize > 1) cluster_sync_all();   // the peer's barriers exist before anyone arrives on them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
@@ -601,11 +601,11 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
         if (lane == 0) {
             const uint64_t pol_keep = policy_evict_last(), pol_drop = policy_evict_first();
             uint32_t it = 0, s = 0, ph = 0;   // F chunks requested so far; ring slot and phase of the next one
-            for (int u = cid; u < p.units; u += nclusters) {
+            for (int u = cid; u < p.units; u += nctas) {
                 const Unit un = decode_unit(p, u);
                 for (int pass = 0; pass < 2; ++pass)
                     for (int g = 0; g < G; ++g) {
-                        const int cg = (g_off + (pass == 0 ? g : G - 1 - g)) * p.gc;
+                        const int cg = (pass == 0 ? g : G - 1 - g) * p.gc;
                         const int nsub = min(p.gc, CT - cg);
                         for (int j = 0; j < nsub; ++j, ++it) {
                             if (!mbar_wait(bar.empty + 8 * s, ph ^ 1u, abort_flag, 100)) {
@@ -624,11 +624,11 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
         // ------------------------------------------------ TMA producer: basis slices ---
         if (lane == 0) {
             uint32_t iv = 0, vs = 0, vph = 0;
-            for (int u = cid; u < p.units; u += nclusters) {
+            for (int u = cid; u < p.units; u += nctas) {
                 const Unit un = decode_unit(p, u);
                 for (int pass = 0; pass < 2; ++pass)
                     for (int g = 0; g < G; ++g, ++iv) {
-                        const int cg = (g_off + (pass == 0 ? g : G - 1 - g)) * p.gc;
+                        const int cg = (pass == 0 ? g : G - 1 - g) * p.gc;
                         if (!mbar_wait(bar.v_empty + 8 * vs, vph ^ 1u, abort_flag, 101)) {
                             record_timeout(p, abort_flag, iv, (uint32_t)(pass * 100 + g));
                             goto done;
@@ -655,10 +655,10 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
             const uint32_t idesc1 = idesc_bf16(kTileRows, p.k);
             const int ksteps = p.kb_elems / 16;
             const uint64_t a_desc0 = smem_desc_kmajor(a_base, p.kb_bytes);
-            for (int u = cid; u < p.units; u += nclusters, ++ui) {
+            for (int u = cid; u < p.units; u += nctas, ++ui) {
                 // C of the previous unit has been read out of TMEM: a_full(ui - 1) was awaited below
                 for (int g = 0; g < G; ++g, ++iv) {                 // pass 1: C_a += F_chunk (V^T chunk)^T
-                    const int cg = (g_off + g) * p.gc, ce = min(cg + p.gc, CT);
+                    const int cg = g * p.gc, ce = min(cg + p.gc, CT);
                     const uint32_t vs = vr.idx;
                     SVDC_TRACE_MARK(t0);
                     if (!mbar_wait(bar.v_full + 8 * vs, vr.ph, abort_flag, 9)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
@@ -675,7 +675,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                         const uint64_t vd = smem_desc_kmajor(v_base0 + vs * p.vslice_bytes + (c - cg) * (p.k * 128), 128);
 #pragma unroll
                         for (int ks = 0; ks < kTileCols / 16; ++ks)
-                            mma_bf16_ss(tmem_base, fd + 2 * ks, vd + 2 * ks, idesc1, (c != c_first || ks != 0) ? 1u : 0u);
+                            mma_bf16_ss(tmem_base, fd + 2 * ks, vd + 2 * ks, idesc1, (c != 0 || ks != 0) ? 1u : 0u);
                         mma_commit(bar.empty + 8 * s);
                         mbar_arrive_n(bar.empty + 8 * s, 4);   // pass 1 has no slab stores: the other four arrivals
                         SVDC_TRACE_ADD(2, t2);
@@ -688,7 +688,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                 SVDC_TRACE_ADD(3, t3);
                 tc_fence_after();
                 for (int g = 0; g < G; ++g, ++iv, ++ig) {           // pass 2: acc = C (V slice)^T
-                    const int cg = (g_off + G - 1 - g) * p.gc;
+                    const int cg = (G - 1 - g) * p.gc;
                     const int nsub = min(p.gc, CT - cg);
                     const uint32_t vs = vr.idx, as = ar.idx;
                     SVDC_TRACE_MARK(t4);
@@ -760,7 +760,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
             const Unit x = decode_unit(p, cid);
             if (*(volatile uint32_t *)&header_of(p, x.b)->full_steps != 0) request_chat(x);
         }
-        for (int u = cid; u < p.units; u += nclusters, ++ui) {
+        for (int u = cid; u < p.units; u += nctas, ++ui) {
             const Unit un = decode_unit(p, u);
             if constexpr (c_split) {
                 // ---- C job, operand in tensor memory (k >= 64): both epilogue groups take part.  Of
@@ -848,14 +848,6 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                     if (kb > 0) load_prev(kb, prev0);
                     k_block(kb, prev0);
                 }
-                // count this unit; the last unit of a block to get here counts the full step
-                if (issuer) {
-                    const uint32_t prevc = atomicAdd(&hdr->done, 1u);
-                    if (prevc == (uint32_t)p.row_tiles - 1u) {
-                        hdr->done = 0;
-                        hdr->full_steps = hdr->full_steps + 1;
-                    }
-                }
             } else if (c_warp) {   // (discarded statement of the if constexpr above when the operand is in TMEM)
                 // ---- C job: TMEM -> EMA -> Chat, split-bf16 A operand (+ the state's operand copy)
                 StateHeader *hdr = header_of(p, un.b);
@@ -871,33 +863,8 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                 tc_fence_after();
                 SVDC_TRACE_MARK(c2);
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-                if constexpr (kClusterSplit) {
-                    // Exchange of the partial C's.  My pass-1 MMAs are complete, hence (the tensor
-                    // pipe runs in order) so are the pass-2 MMAs of my previous unit: my A region
-                    // is free, and I tell the peer so.  Once the peer has said the same, every C
-                    // thread writes its row of my partial into the peer's A region (the layout of
-                    // the staged Chat: 32-column blocks of 128-byte swizzled rows) and arrives on
-                    // the peer's recv_full; my own recv_full then says the peer's partial is here.
-                    const uint32_t peer = crank ^ 1u;
-                    if (issuer) mbar_arrive_remote(mapa_shared(peer_ready, peer));
-                    bool okx = mbar_wait_cluster(peer_ready, ui & 1u, abort_flag, 20);
-                    if (!__all_sync(0xFFFFFFFFu, okx)) { record_timeout(p, abort_flag, it, ig, ui); goto done; }
-                    for (int b = 0; b < nblk; ++b) {
-                        uint32_t tmp[32];
-                        tmem_ld_32x32(taddr + b * 32, tmp);
-                        tmem_wait_ld();
-                        const uint32_t rrow = mapa_shared(a_base + (uint32_t)b * kBlk32Bytes + (uint32_t)row * 128u, peer);
-#pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            st_cluster128(rrow + (((uint32_t)i) ^ ((uint32_t)row & 7u)) * 16u,
-                                          make_uint4(tmp[4 * i], tmp[4 * i + 1], tmp[4 * i + 2], tmp[4 * i + 3]));
-                    }
-                    mbar_arrive_remote(mapa_shared(recv_full, peer));
-                    okx = mbar_wait_cluster(recv_full, ui & 1u, abort_flag, 21);
-                    if (!__all_sync(0xFFFFFFFFu, okx)) { record_timeout(p, abort_flag, it, ig, ui); goto done; }
-                }
                 const int64_t n = (int64_t)un.rt * kTileRows + row;
-                const bool row_live = n < p.N && crank == 0;   // in a cluster, rank 0 writes the coefficient arrays
+                const bool row_live = n < p.N;
                 char *st_b = p.state + (size_t)un.b * p.state_stride;
                 float *chat_g = reinterpret_cast<float *>(st_b + p.chat_off) + n * p.k;
                 float *cout_g = p.C_out ? reinterpret_cast<float *>((char *)p.C_out + (size_t)un.b * p.C_stride) + n * p.k
@@ -914,10 +881,6 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                     const int halves = p.k >= 64 ? 2 : 1;
                     float prevB[32];
                     if (!first && halves == 2) load_row32(stB, (uint32_t)row, chat_row_bytes, 32, prevB);
-                    // cluster mode: the peer's partial sits where this row's hi / lo operand rows go
-                    // (the staged Chat has a buffer of its own then); read the lo half's block first
-                    float recvB[kClusterSplit ? 32 : 1];
-                    if constexpr (kClusterSplit) load_row32(lo_row, (uint32_t)row, 128u, 32, recvB);
                     for (int h = 0; h < halves; ++h) {
                         const int col0 = kb * 64 + h * 32;
                         const int ncols = p.k - col0 < 32 ? p.k - col0 : 32;
@@ -928,17 +891,6 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                             tmem_wait_ld();
 #pragma unroll
                             for (int i = 0; i < 32; ++i) cs[i] = __uint_as_float(tmp[i]);
-                        }
-                        if constexpr (kClusterSplit) {   // C = my partial + the peer's (a + b == b + a: both CTAs get the same bits)
-                            if (h == 0) {
-                                float recvA[32];
-                                load_row32(hi_row, (uint32_t)row, 128u, 32, recvA);
-#pragma unroll
-                                for (int i = 0; i < 32; ++i) cs[i] += recvA[i];
-                            } else {
-#pragma unroll
-                                for (int i = 0; i < 32; ++i) cs[i] += recvB[i];
-                            }
                         }
                         float ch[32];
                         if (first) {
@@ -994,22 +946,14 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                 fence_proxy_async();
                 mbar_arrive(bar.a_full);
                 SVDC_TRACE_ADD(2, c2);
-                // count this unit; the last unit of a block to get here counts the full step
-                if (issuer && crank == 0) {
-                    const uint32_t prev = atomicAdd(&hdr->done, 1u);
-                    if (prev == (uint32_t)p.row_tiles - 1u) {
-                        hdr->done = 0;
-                        hdr->full_steps = hdr->full_steps + 1;
-                    }
-                }
             }
             // ---- epilogue duty for this group's chunks of pass 2
             const int slab_row0 = un.rt * kTileRows + q * kSlabRows;
             const bool slab_live = (int64_t)slab_row0 < p.N;
-            it += CTm;   // pass-1 slots are consumed by the MMA warp alone
-            fr.skip((uint32_t)CTm, (uint32_t)p.stages);
+            it += CT;   // pass-1 slots are consumed by the MMA warp alone
+            fr.skip((uint32_t)CT, (uint32_t)p.stages);
             for (int g = 0; g < G; ++g, ++ig) {
-                const int cg = (g_off + G - 1 - g) * p.gc;
+                const int cg = (G - 1 - g) * p.gc;
                 const int nsub = min(p.gc, CT - cg);
                 const uint32_t as = ar.idx, aph = ar.ph;
                 ar.step((uint32_t)p.acc_stages);
@@ -1076,7 +1020,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
             // Every accumulator of this unit has been read, so its pass-2 MMAs are complete and
             // the A region is free: stage the next unit's previous Chat there.
             if (issuer) {
-                const int un_next = u + nclusters;
+                const int un_next = u + nctas;
                 const bool ok = mbar_wait(p2_done, ui & 1u, abort_flag, 18);
                 if (ok && un_next < p.units && !c_split) {
                     const Unit x = decode_unit(p, un_next);
@@ -1092,572 +1036,29 @@ done:
     SVDC_TRACE_FLUSH(g_trace);
     tc_fence_before();
     __syncthreads();
-    if (csize > 1) cluster_sync_all();   // no CTA leaves while its peer may still reach into it
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, tmem_cols);
     }
+    if (threadIdx.x == 0) report_exit_and_count_step(p);
 }
 
-// ======================================================================================
-// Full step, batched two-phase schedule (Eq. 8 - Eq. 11)
-//
-// The one-CTA-per-tile kernel above keeps 148 tiles (113 MB of F at D = 3072) between its
-// two passes, more than L2 holds next to the R write stream.  Here the tiles are taken in
-// batches of Bt = grid / Q, and every tile of a batch is shared by Q CTAs, one column slice
-// each.  CTA c = (tile-in-batch, slice) runs, for batch b = 0, 1, ...:
-//   P1(b):   its slice of C = F V_k for its tile of batch b, into a TMEM accumulator; the dump
-//            warps write that partial C (fp32) into the head of the tile's R rows -- R is about
-//            to be overwritten by this very step -- and count the tile's arrivals; the last
-//            of the Q slices to arrive combines them in slice order (so the sum does not
-//            depend on timing), applies the EMA, writes Chat, its operand copy, C_out and C
-//            as a split-bf16 pair into the state's scratch, and marks the tile ready;
-//   P2(b-1): its slice of R = F - C V_k^T for its tile of the previous batch, exactly like the
-//            cached step: the A operand (split C) comes by TMA once the tile is marked ready,
-//            which it has long been, F is read again (two batches of F stay in flight: 57 MB
-//            at D = 3072, an L2 hit), and the epilogue stores R.
-// Nothing serial sits between the passes of a CTA any more: the combination of batch b runs
-// on warps of its own while P2(b-1) streams.
-//
-// Warp roles (448 threads): 0 = TMA producer, 1 = MMA issuer (+ TMEM owner), 2..9 = two
-// epilogue groups, 10..13 = dump / combine.
-// TMEM: two C accumulators in columns [0, 2k), then the pass-2 accumulator ring.
-// ======================================================================================
-constexpr int kThreadsFull2 = 448;
-
-struct Bars2 {
-    uint32_t full, empty, v_full, v_empty, acc_full, acc_empty, c_full, c_empty, a_full, a_empty, tmem_slot, abort_flag, last_flag;
-};
-__device__ __forceinline__ Bars2 bars2_at(uint32_t base) {
-    Bars2 b;
-    b.full = base;
-    b.empty = b.full + 8 * kMaxStages;
-    b.v_full = b.empty + 8 * kMaxStages;
-    b.v_empty = b.v_full + 8 * kMaxVSlots;
-    b.acc_full = b.v_empty + 8 * kMaxVSlots;
-    b.acc_empty = b.acc_full + 8 * kAccStages;
-    b.c_full = b.acc_empty + 8 * kAccStages;
-    b.c_empty = b.c_full + 16;
-    b.a_full = b.c_empty + 16;
-    b.a_empty = b.a_full + 8;
-    b.tmem_slot = b.a_empty + 8;
-    b.abort_flag = b.tmem_slot + 8;
-    b.last_flag = b.abort_flag + 8;
-    return b;
-}
-constexpr uint32_t kBar2Bytes = 8 * (2 * kMaxStages + 2 * kMaxVSlots + 2 * kAccStages + 2 + 2 + 2 + 3);
-
-struct Unit2 {
-    int valid, blk, rt, tile, g_off, G, c_first, nchunks;   // tile = index among all tiles of the launch
-};
-// unit of CTA `cta` in batch b (P1 of batch b, P2 of batch b one iteration later)
-__device__ __forceinline__ Unit2 unit2_of(const UmmaParams &p, int cta, int b, int G_all) {
-    Unit2 u;
-    const int tib = cta / p.Q, dq = cta - tib * p.Q;
-    u.tile = b * p.Bt + tib;
-    u.valid = (b >= 0 && b < p.nbat && tib < p.Bt && u.tile < p.T) ? 1 : 0;
-    u.blk = u.tile / p.row_tiles;
-    u.rt = u.tile - u.blk * p.row_tiles;
-    u.g_off = (dq * G_all) / p.Q;
-    u.G = ((dq + 1) * G_all) / p.Q - u.g_off;
-    u.c_first = u.g_off * p.gc;
-    u.nchunks = min(p.chunks_total, (u.g_off + u.G) * p.gc) - u.c_first;
-    return u;
-}
-__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *ptr) {
-    uint32_t v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
-    return v;
-}
-__device__ __forceinline__ void st_release_u32(uint32_t *ptr, uint32_t v) {
-    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(ptr), "r"(v) : "memory");
-}
-__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
-
-__global__ void __launch_bounds__(kThreadsFull2, 1)
-umma_full2_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant__ CUtensorMap tm_vt,
-                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_rout,
-                  const __grid_constant__ CUtensorMap tm_chi, const __grid_constant__ CUtensorMap tm_clo,
-                  const UmmaParams p) {
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t a_base = base;                                  // split C operand of the P2 unit (hi | lo)
-    const uint32_t v_base0 = a_base + p.a_bytes;
-    const uint32_t stage0 = v_base0 + (uint32_t)p.v_slots * p.vslice_bytes;
-    const Bars2 bar = bars2_at(stage0 + (uint32_t)p.stages * kTileBytes);
-    uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(gen_base + (bar.abort_flag - base));
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(gen_base + (bar.tmem_slot - base));
-    volatile int *last_flag = reinterpret_cast<volatile int *>(gen_base + (bar.last_flag - base));
-
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    SVDC_TRACE_DECL
-    const int cta = (int)blockIdx.x;
-    const int CT = p.chunks_total;
-    const int G_all = (CT + p.gc - 1) / p.gc;
-    const uint32_t ring_col = 2u * (uint32_t)p.k;   // first TMEM column of the pass-2 ring
-
+// One CTA that waits, with the bounded wait of the step kernels, for an mbarrier phase nobody
+// will ever complete: the wait must give up after `limit` cycles, the kernel must record the
+// time-out in the state header exactly as the step kernels do, and return.
+__global__ void __launch_bounds__(64, 1) wait_selftest_kernel(const UmmaParams p, long long limit) {
+    __shared__ __align__(8) unsigned long long bar_mem;
+    __shared__ int abort_mem;
+    const uint32_t bar = smem_u32(&bar_mem);
+    volatile int *abort_flag = &abort_mem;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < p.stages; ++s) { mbar_init(bar.full + 8 * s, 1); mbar_init(bar.empty + 8 * s, 5); }
-        for (int s = 0; s < p.v_slots; ++s) { mbar_init(bar.v_full + 8 * s, 1); mbar_init(bar.v_empty + 8 * s, 1); }
-        for (int s = 0; s < p.acc_stages; ++s) { mbar_init(bar.acc_full + 8 * s, 1); mbar_init(bar.acc_empty + 8 * s, 8); }
-        for (int s = 0; s < 2; ++s) { mbar_init(bar.c_full + 8 * s, 1); mbar_init(bar.c_empty + 8 * s, 128); }
-        mbar_init(bar.a_full, 1);
-        mbar_init(bar.a_empty, 1);
-        *abort_flag = 0;
-        *last_flag = 0;
+        mbar_init(bar, 1);
+        abort_mem = 0;
         fence_barrier_init();
-        prefetch_tensormap(&tm_f);
-        prefetch_tensormap(&tm_vt);
-        prefetch_tensormap(&tm_v);
-        prefetch_tensormap(&tm_rout);
-        prefetch_tensormap(&tm_chi);
-        prefetch_tensormap(&tm_clo);
     }
-    if (warp == 1) {
-        tmem_alloc(bar.tmem_slot, 512);
-        tmem_relinquish();
-    }
-    tc_fence_before();
     __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
-
-    if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer ---
-        // Three request streams polled without blocking: basis slices and F chunks in the order
-        // P1(0), P1(1), P2(0), P1(2), P2(1), ..., and the A operand of each P2 unit, which also
-        // has to wait for the tile's ready mark.
-        if (lane == 0) {
-            const uint64_t pol_keep = policy_evict_last(), pol_drop = policy_evict_first();
-            struct Step { int b, phase, g; };   // phase 0 = P1 of batch b, 1 = P2 of batch b - lag
-            auto step_unit = [&](const Step &x) { return unit2_of(p, cta, x.phase == 0 ? x.b : x.b - p.lag, G_all); };
-            auto normalise = [&](Step x) {      // skip (batch, phase) pairs this CTA has no unit for
-                while (x.b < p.nbat + p.lag) {
-                    const Unit2 u = step_unit(x);
-                    if (u.valid && x.g < u.G) return x;
-                    x.g = 0;
-                    if (++x.phase == 2) { x.phase = 0; ++x.b; }
-                }
-                return x;
-            };
-            auto advance = [&](Step x) { ++x.g; return normalise(x); };
-            Step vcur = normalise(Step{0, 0, 0}), fcur = vcur;
-            int fc = 0;
-            uint32_t iv = 0, it = 0;   // basis slices, F chunks requested so far
-            long long t_idle = clock64();
-            while (fcur.b < p.nbat + p.lag || vcur.b < p.nbat + p.lag) {
-                bool progress = false;
-                if (vcur.b < p.nbat + p.lag) {
-                    const uint32_t vs = iv % p.v_slots;
-                    if (mbar_test_wait(bar.v_empty + 8 * vs, ((iv / p.v_slots) & 1u) ^ 1u)) {
-                        const Unit2 u = step_unit(vcur);
-                        const int cg = (u.g_off + (vcur.phase == 0 ? vcur.g : u.G - 1 - vcur.g)) * p.gc;
-                        const uint32_t vdst = v_base0 + vs * p.vslice_bytes;
-                        mbar_arrive_expect_tx(bar.v_full + 8 * vs, p.vslice_bytes);
-                        if (vcur.phase == 0) {
-                            for (int j = 0; j < p.gc; ++j)
-                                tma_load_3d(vdst + j * (p.k * 128), &tm_vt, bar.v_full + 8 * vs, (cg + j) * kTileCols, 0, u.blk);
-                        } else {
-                            for (int kb = 0; kb < p.nkb; ++kb)
-                                tma_load_3d(vdst + kb * (p.gc * kTileCols * p.kb_bytes), &tm_v, bar.v_full + 8 * vs,
-                                            kb * p.kb_elems, cg * kTileCols, u.blk);
-                        }
-                        vcur = advance(vcur);
-                        ++iv;
-                        progress = true;
-                    }
-                }
-                if (fcur.b < p.nbat + p.lag) {
-                    const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                    if (mbar_test_wait(bar.empty + 8 * s, ph ^ 1u)) {
-                        const Unit2 u = step_unit(fcur);
-                        const int cg = (u.g_off + (fcur.phase == 0 ? fcur.g : u.G - 1 - fcur.g)) * p.gc;
-                        const int nsub = min(p.gc, CT - cg);
-                        mbar_arrive_expect_tx(bar.full + 8 * s, kTileBytes);
-                        tma_load_3d_hint(stage0 + s * kTileBytes, &tm_f, bar.full + 8 * s, (cg + fc) * kTileCols,
-                                         u.rt * kTileRows, u.blk, fcur.phase == 0 ? pol_keep : pol_drop);
-                        ++it;
-                        if (++fc == nsub) { fc = 0; fcur = advance(fcur); }
-                        progress = true;
-                    }
-                }
-                if (progress) {
-                    t_idle = clock64();
-                } else if (*abort_flag || clock64() - t_idle > kWaitCycles) {
-                    atomicCAS(const_cast<int *>(abort_flag), 0, 100);
-                    record_timeout(p, abort_flag, it, iv, 0);
-                    goto done;
-                }
-            }
-        } else if (lane == 1) {
-            // The A operand of each P2 unit (split C of its tile): requested once the previous P2
-            // unit's MMAs have released the buffer and the tile carries this step's ready mark.
-            // A thread of its own, so that polling the mark (a global load) never slows the
-            // other two request streams down.
-            uint32_t na = 0;
-            for (int b = 0; b < p.nbat; ++b) {
-                const Unit2 u = unit2_of(p, cta, b, G_all);
-                if (!u.valid) continue;
-                char *st_b = p.state + (size_t)u.blk * p.state_stride;
-                const uint32_t want = *(volatile uint32_t *)&reinterpret_cast<StateHeader *>(st_b)->full_steps + 1u;
-                const uint32_t *ready = reinterpret_cast<const uint32_t *>(st_b + p.sync_off) + 4 * u.rt + 2;
-                if (!mbar_wait(bar.a_empty, (na & 1u) ^ 1u, abort_flag, 40)) { record_timeout(p, abort_flag, na, (uint32_t)b, 0); break; }
-                const long long t0 = clock64();
-                bool ok = true;
-                while (ld_acquire_u32(ready) != want) {
-                    __nanosleep(200);
-                    if (*abort_flag || clock64() - t0 > kWaitCycles) { atomicCAS(const_cast<int *>(abort_flag), 0, 41); ok = false; break; }
-                }
-                if (!ok) { record_timeout(p, abort_flag, na, (uint32_t)b, 1); break; }
-                fence_proxy_async_all();   // the pair was written with ordinary stores by other SMs
-                mbar_arrive_expect_tx(bar.a_full, p.a_bytes);
-                for (int kb = 0; kb < p.nkb; ++kb) {
-                    tma_load_3d(a_base + kb * (kTileRows * p.kb_bytes), &tm_chi, bar.a_full, kb * p.kb_elems,
-                                u.rt * kTileRows, u.blk);
-                    tma_load_3d(a_base + p.a_half_bytes + kb * (kTileRows * p.kb_bytes), &tm_clo, bar.a_full,
-                                kb * p.kb_elems, u.rt * kTileRows, u.blk);
-                }
-                ++na;
-            }
-        }
-    } else if (warp == 1) {
-        // -------------------------------------------------------------- MMA issuer ---
-        if (lane == 0) {
-            uint32_t it = 0, iv = 0, ig = 0, n1 = 0, n2 = 0;   // F chunks, basis slices, P2 groups, P1 units, P2 units
-            const uint32_t idesc1 = idesc_bf16(kTileRows, p.k);
-            const int ksteps = p.kb_elems / 16;
-            const uint64_t a_desc0 = smem_desc_kmajor(a_base, p.kb_bytes);
-            for (int b = 0; b < p.nbat + p.lag; ++b) {
-                const Unit2 u1 = unit2_of(p, cta, b, G_all);
-                if (u1.valid) {                                  // ---- P1(b): C slice into accumulator n1 & 1
-                    const uint32_t ci = n1 & 1u;
-                    SVDC_TRACE_MARK(m0);
-                    if (!mbar_wait(bar.c_empty + 8 * ci, ((n1 >> 1) & 1u) ^ 1u, abort_flag, 30)) { record_timeout(p, abort_flag, it, iv, n1); goto done; }
-                    SVDC_TRACE_ADD(0, m0);
-                    tc_fence_after();
-                    for (int g = 0; g < u1.G; ++g, ++iv) {
-                        const int cg = (u1.g_off + g) * p.gc, ce = min(cg + p.gc, CT);
-                        const uint32_t vs = iv % p.v_slots;
-                        SVDC_TRACE_MARK(m1);
-                        if (!mbar_wait(bar.v_full + 8 * vs, (iv / p.v_slots) & 1u, abort_flag, 31)) { record_timeout(p, abort_flag, it, iv, n1); goto done; }
-                        SVDC_TRACE_ADD(1, m1);
-                        for (int c = cg; c < ce; ++c, ++it) {
-                            const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                            SVDC_TRACE_MARK(m1b);
-                            if (!mbar_wait(bar.full + 8 * s, ph, abort_flag, 32)) { record_timeout(p, abort_flag, it, iv, n1); goto done; }
-                            SVDC_TRACE_ADD(1, m1b);
-                            tc_fence_after();
-                            SVDC_TRACE_MARK(m2);
-                            const uint64_t fd = smem_desc_kmajor(stage0 + s * kTileBytes, 128);
-                            const uint64_t vd = smem_desc_kmajor(v_base0 + vs * p.vslice_bytes + (c - cg) * (p.k * 128), 128);
-#pragma unroll
-                            for (int ks = 0; ks < kTileCols / 16; ++ks)
-                                mma_bf16_ss(tmem_base + ci * p.k, fd + 2 * ks, vd + 2 * ks, idesc1, (c != u1.c_first || ks != 0) ? 1u : 0u);
-                            mma_commit(bar.empty + 8 * s);
-                            mbar_arrive_n(bar.empty + 8 * s, 4);   // pass 1 has no slab stores: the other four arrivals
-                            SVDC_TRACE_ADD(2, m2);
-                        }
-                        mma_commit(bar.v_empty + 8 * vs);
-                    }
-                    mma_commit(bar.c_full + 8 * ci);
-                    ++n1;
-                }
-                const Unit2 u2 = unit2_of(p, cta, b - p.lag, G_all);
-                if (u2.valid) {                                  // ---- P2(b - lag): acc = C (V slice)^T
-                    SVDC_TRACE_MARK(m3);
-                    if (!mbar_wait(bar.a_full, n2 & 1u, abort_flag, 33)) { record_timeout(p, abort_flag, it, iv, n2); goto done; }
-                    SVDC_TRACE_ADD(3, m3);
-                    tc_fence_after();
-                    for (int g = 0; g < u2.G; ++g, ++iv, ++ig) {
-                        const int cg = (u2.g_off + u2.G - 1 - g) * p.gc;
-                        const int nsub = min(p.gc, CT - cg);
-                        const uint32_t vs = iv % p.v_slots, as = ig % p.acc_stages;
-                        SVDC_TRACE_MARK(m4);
-                        if (!mbar_wait(bar.v_full + 8 * vs, (iv / p.v_slots) & 1u, abort_flag, 34)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
-                        SVDC_TRACE_ADD(4, m4);
-                        SVDC_TRACE_MARK(m5);
-                        if (!mbar_wait(bar.acc_empty + 8 * as, ((ig / p.acc_stages) & 1u) ^ 1u, abort_flag, 35)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
-                        SVDC_TRACE_ADD(5, m5);
-                        tc_fence_after();
-                        const uint32_t idesc = idesc_bf16(kTileRows, nsub * kTileCols);
-                        const uint32_t d_tmem = tmem_base + ring_col + as * p.acc_cols;
-                        const uint64_t v_desc0 = smem_desc_kmajor(v_base0 + vs * p.vslice_bytes, p.kb_bytes);
-                        uint32_t acc = 0;
-                        for (int part = 0; part < 2; ++part)
-                            for (int kb = 0; kb < p.nkb; ++kb) {
-                                const uint64_t ad = a_desc0 + ((part * p.a_half_bytes + kb * (kTileRows * p.kb_bytes)) >> 4);
-                                const uint64_t vd = v_desc0 + ((kb * (p.gc * kTileCols * p.kb_bytes)) >> 4);
-                                for (int ks = 0; ks < ksteps; ++ks) {
-                                    mma_bf16_ss(d_tmem, ad + 2 * ks, vd + 2 * ks, idesc, acc);
-                                    acc = 1;
-                                }
-                            }
-                        mma_commit(bar.v_empty + 8 * vs);
-                        mma_commit(bar.acc_full + 8 * as);
-                        // see every phase of the F slots of pass 2 as well, and gate their reuse
-                        SVDC_TRACE_MARK(m6);
-                        for (int j = 0; j < nsub; ++j, ++it) {
-                            const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                            if (!mbar_wait(bar.full + 8 * s, ph, abort_flag, 36)) { record_timeout(p, abort_flag, it, iv, ig); goto done; }
-                            mbar_arrive(bar.empty + 8 * s);
-                        }
-                        SVDC_TRACE_ADD(6, m6);
-                    }
-                    mma_commit(bar.a_empty);
-                    ++n2;
-                }
-            }
-        }
-    } else if (warp < 10) {
-        // ------------------------------------------- epilogue of the P2 units: R = F - C V_k^T ---
-        const int q = warp & 3, row = q * kSlabRows + lane;
-        const uint32_t grp = (uint32_t)(warp - 2) >> 2;
-        uint32_t it = 0, ig = 0;
-        int prev_slot = -1;
-        const bool defer_release = p.stages >= 4;
-        for (int b = 0; b < p.nbat + p.lag; ++b) {
-            const Unit2 u1 = unit2_of(p, cta, b, G_all);
-            if (u1.valid) it += u1.nchunks;   // pass-1 slots are consumed by the MMA warp alone
-            const Unit2 u2 = unit2_of(p, cta, b - p.lag, G_all);
-            if (!u2.valid) continue;
-            const int slab_row0 = u2.rt * kTileRows + q * kSlabRows;
-            const bool slab_live = (int64_t)slab_row0 < p.N;
-            for (int g = 0; g < u2.G; ++g, ++ig) {
-                const int cg = (u2.g_off + u2.G - 1 - g) * p.gc;
-                const int nsub = min(p.gc, CT - cg);
-                const uint32_t as = ig % p.acc_stages, aph = (ig / p.acc_stages) & 1u;
-                const int last_own = last_own_chunk(it, nsub, grp);
-                SVDC_TRACE_MARK(e0);
-                if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar.acc_full + 8 * as, aph, abort_flag, 37))) { record_timeout(p, abort_flag, it, ig, b); goto done; }
-                SVDC_TRACE_ADD(0, e0);
-                if (last_own < 0 && lane == 0) mbar_arrive(bar.acc_empty + 8 * as);
-                for (int j = 0; j < nsub; ++j, ++it) {
-                    if ((it & 1u) != grp) continue;
-                    const int c = cg + j;
-                    const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                    SVDC_TRACE_MARK(e1);
-                    if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar.full + 8 * s, ph, abort_flag, 38))) { record_timeout(p, abort_flag, it, ig, b); goto done; }
-                    SVDC_TRACE_ADD(1, e1);
-                    tc_fence_after();
-                    SVDC_TRACE_MARK(e2);
-                    const uint32_t tile = stage0 + s * kTileBytes + (uint32_t)row * 128u;
-                    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + ring_col + as * p.acc_cols + j * kTileCols;
-                    uint32_t acc0[32], acc1[32];
-                    tmem_ld_32x32(taddr, acc0);
-                    tmem_ld_32x32(taddr + 32, acc1);
-                    uint4 t[8];
-#pragma unroll
-                    for (int cc = 0; cc < 8; ++cc) t[cc] = lds128(tile + (((uint32_t)cc) ^ ((uint32_t)row & 7u)) * 16u);
-                    tmem_wait_ld();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0 && j == last_own) mbar_arrive(bar.acc_empty + 8 * as);
-#pragma unroll
-                    for (int cc = 0; cc < 8; ++cc)
-                        sts128(tile + (((uint32_t)cc) ^ ((uint32_t)row & 7u)) * 16u,
-                               combine_chunk<true>(t[cc], cc < 4 ? acc0 + cc * 8 : acc1 + (cc - 4) * 8));
-                    fence_proxy_async();
-                    __syncwarp();
-                    if (lane == 0) {
-                        if (slab_live)
-                            tma_store_3d(&tm_rout, stage0 + s * kTileBytes + (uint32_t)q * kSlabBytes, c * kTileCols,
-                                         slab_row0, u2.blk);
-                        tma_store_commit();
-                        if (!defer_release) {
-                            tma_store_wait_read<0>();
-                            mbar_arrive(bar.empty + 8 * s);
-                        } else {
-                            if (prev_slot >= 0) {
-                                tma_store_wait_read<1>();
-                                mbar_arrive(bar.empty + 8 * prev_slot);
-                            }
-                            prev_slot = (int)s;
-                        }
-                    }
-                    __syncwarp();
-                    SVDC_TRACE_ADD(2, e2);
-                    SVDC_TRACE_COUNT(3);
-                }
-            }
-            if (lane == 0 && prev_slot >= 0) {
-                tma_store_wait_read<0>();
-                mbar_arrive(bar.empty + 8 * prev_slot);
-                prev_slot = -1;
-            }
-            // count the unit; the last P2 unit of a block counts the full step (nobody of this
-            // launch reads the counter of that block afterwards)
-            if (warp == 2 && lane == 0) {
-                StateHeader *hdr = header_of(p, u2.blk);
-                const uint32_t prev = atomicAdd(&hdr->done, 1u);
-                if (prev == (uint32_t)(p.row_tiles * p.Q) - 1u) {
-                    hdr->done = 0;
-                    hdr->full_steps = hdr->full_steps + 1;
-                }
-            }
-        }
-        if (lane == 0) tma_store_wait<0>();
-    } else {
-        // ------------------ dump of the partial C, then the combination of this CTA's share of rows ---
-        // sync words of a tile: [0] slices dumped, [1] row shares combined, [2] ready mark (= full
-        // steps seen + 1).  The Q slice CTAs of a tile each combine 128 / Q of its rows once all Q
-        // partials are there, in slice order, so the sums do not depend on timing; the last share
-        // to finish resets the counters and sets the mark.
-        const int q = warp & 3, row = q * 32 + lane, tid = threadIdx.x - 320;
-        const float beta = p.beta, omb = 1.0f - p.beta;
-        const int nblk = (p.k + 31) / 32;
-        const int dq = cta % p.Q;
-        const int share = kTileRows / p.Q;               // rows this CTA combines (Q is 1, 2, 4 or 8)
-        const int tpr = 128 / share;                      // threads per row in the combination
-        const int cols_pt = p.k / tpr;                    // columns per thread there (k / tpr, a multiple of 4)
-        uint32_t n1 = 0;
-        bool dead = false;   // a wait ran out: skip all work but keep the named barriers in step
-        for (int b = 0; b < p.nbat; ++b) {
-            const Unit2 u = unit2_of(p, cta, b, G_all);
-            if (!u.valid) continue;
-            const uint32_t ci = n1 & 1u;
-            char *st_b = p.state + (size_t)u.blk * p.state_stride;
-            StateHeader *hdr = reinterpret_cast<StateHeader *>(st_b);
-            uint32_t *sync = reinterpret_cast<uint32_t *>(st_b + p.sync_off) + 4 * u.rt;
-            const int64_t n = (int64_t)u.rt * kTileRows + row;
-            // partial C's of the tile: Q x k floats at the head of each of its R rows
-            char *r_rows = st_b + p.r_off;
-            SVDC_TRACE_MARK(d0);
-            if (!dead && !__all_sync(0xFFFFFFFFu, mbar_wait(bar.c_full + 8 * ci, (n1 >> 1) & 1u, abort_flag, 39))) {
-                record_timeout(p, abort_flag, n1, (uint32_t)b, 0);
-                dead = true;
-            }
-            SVDC_TRACE_ADD(0, d0);
-            SVDC_TRACE_MARK(d1);
-            ++n1;
-            if (!dead) {
-                tc_fence_after();
-                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + ci * p.k;
-                float *scratch_row = reinterpret_cast<float *>(r_rows + (size_t)n * p.D * 2);
-                for (int cb = 0; cb < nblk; ++cb) {
-                    uint32_t tmp[32];
-                    tmem_ld_32x32(taddr + cb * 32, tmp);
-                    tmem_wait_ld();
-                    const int ncols = min(32, p.k - cb * 32);
-                    if (n < p.N) {
-#pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            if (i * 4 < ncols)
-                                __stcg(reinterpret_cast<uint4 *>(scratch_row + dq * p.k + cb * 32 + 4 * i),
-                                       make_uint4(tmp[4 * i], tmp[4 * i + 1], tmp[4 * i + 2], tmp[4 * i + 3]));
-                    }
-                }
-                tc_fence_before();
-                mbar_arrive(bar.c_empty + 8 * ci);   // the accumulator may be reused
-                __threadfence();
-            }
-            SVDC_TRACE_ADD(1, d1);
-            named_barrier_sync(3, 128);
-            SVDC_TRACE_MARK(d2);
-            if (tid == 0) {
-                int okw = 0;
-                if (!dead) {
-                    atomicAdd(&sync[0], 1u);
-                    const long long t0 = clock64();
-                    okw = 1;
-                    while (ld_acquire_u32(&sync[0]) < (uint32_t)p.Q) {   // all Q partials of the tile
-                        __nanosleep(100);
-                        if (*abort_flag || clock64() - t0 > kWaitCycles) { atomicCAS(const_cast<int *>(abort_flag), 0, 42); okw = 0; break; }
-                    }
-                    if (!okw) record_timeout(p, abort_flag, n1, (uint32_t)b, 2);
-                }
-                *last_flag = okw;
-            }
-            named_barrier_sync(3, 128);
-            if (*last_flag == 0) dead = true;
-            SVDC_TRACE_ADD(2, d2);
-            SVDC_TRACE_MARK(d3);
-            if (!dead) {
-                __threadfence();
-                // ---- combination of rows [dq * share, (dq + 1) * share) of the tile: thread -> (row, columns)
-                const bool first = *(volatile uint32_t *)&hdr->full_steps == 0;
-                const int crow = dq * share + tid / tpr, c_lo = (tid % tpr) * cols_pt;
-                const int64_t cn = (int64_t)u.rt * kTileRows + crow;
-                if (cn < p.N) {
-                    const float *srow = reinterpret_cast<const float *>(r_rows + (size_t)cn * p.D * 2);
-                    float *chat_g = reinterpret_cast<float *>(st_b + p.chat_off) + cn * p.k;
-                    float *cout_g = p.C_out ? reinterpret_cast<float *>((char *)p.C_out + (size_t)u.blk * p.C_stride) + cn * p.k
-                                            : nullptr;
-                    __nv_bfloat16 *ohi = reinterpret_cast<__nv_bfloat16 *>(st_b + p.ophi_off) + cn * p.k;
-                    __nv_bfloat16 *olo = reinterpret_cast<__nv_bfloat16 *>(st_b + p.oplo_off) + cn * p.k;
-                    __nv_bfloat16 *chi = reinterpret_cast<__nv_bfloat16 *>(st_b + p.chi_off) + cn * p.k;
-                    __nv_bfloat16 *clo = reinterpret_cast<__nv_bfloat16 *>(st_b + p.clo_off) + cn * p.k;
-                    for (int c0 = c_lo; c0 < c_lo + cols_pt; c0 += 8) {
-                        const int w = min(8, c_lo + cols_pt - c0);   // 8, or 4 at the tail of a narrow share
-                        float4 x[8][2], pv[2];
-#pragma unroll
-                        for (int d = 0; d < 8; ++d) {
-                            x[d][0] = x[d][1] = make_float4(0.f, 0.f, 0.f, 0.f);
-                            if (d < p.Q) {
-                                x[d][0] = __ldcg(reinterpret_cast<const float4 *>(srow + d * p.k + c0));
-                                if (w > 4) x[d][1] = __ldcg(reinterpret_cast<const float4 *>(srow + d * p.k + c0 + 4));
-                            }
-                        }
-                        pv[0] = pv[1] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        if (!first) {
-                            pv[0] = *reinterpret_cast<const float4 *>(chat_g + c0);
-                            if (w > 4) pv[1] = *reinterpret_cast<const float4 *>(chat_g + c0 + 4);
-                        }
-                        float cs[8];
-#pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            float4 a = x[0][h];
-#pragma unroll
-                            for (int d = 1; d < 8; ++d) { a.x += x[d][h].x; a.y += x[d][h].y; a.z += x[d][h].z; a.w += x[d][h].w; }
-                            cs[4 * h] = a.x; cs[4 * h + 1] = a.y; cs[4 * h + 2] = a.z; cs[4 * h + 3] = a.w;
-                        }
-                        float ch[8];
-                        const float pf[8] = {pv[0].x, pv[0].y, pv[0].z, pv[0].w, pv[1].x, pv[1].y, pv[1].z, pv[1].w};
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) ch[i] = first ? cs[i] : fmaf(beta, pf[i], omb * cs[i]);
-                        uint4 hi, lo, chh, cll;
-                        pack_split8(ch, hi, lo);
-                        pack_split8(cs, chh, cll);
-                        *reinterpret_cast<float4 *>(chat_g + c0) = make_float4(ch[0], ch[1], ch[2], ch[3]);
-                        if (cout_g) *reinterpret_cast<float4 *>(cout_g + c0) = make_float4(cs[0], cs[1], cs[2], cs[3]);
-                        if (w > 4) {
-                            *reinterpret_cast<float4 *>(chat_g + c0 + 4) = make_float4(ch[4], ch[5], ch[6], ch[7]);
-                            if (cout_g) *reinterpret_cast<float4 *>(cout_g + c0 + 4) = make_float4(cs[4], cs[5], cs[6], cs[7]);
-                            *reinterpret_cast<uint4 *>(ohi + c0) = hi;
-                            *reinterpret_cast<uint4 *>(olo + c0) = lo;
-                            *reinterpret_cast<uint4 *>(chi + c0) = chh;
-                            *reinterpret_cast<uint4 *>(clo + c0) = cll;
-                        } else {
-                            *reinterpret_cast<uint2 *>(ohi + c0) = make_uint2(hi.x, hi.y);
-                            *reinterpret_cast<uint2 *>(olo + c0) = make_uint2(lo.x, lo.y);
-                            *reinterpret_cast<uint2 *>(chi + c0) = make_uint2(chh.x, chh.y);
-                            *reinterpret_cast<uint2 *>(clo + c0) = make_uint2(cll.x, cll.y);
-                        }
-                    }
-                }
-                __threadfence();
-            }
-            named_barrier_sync(3, 128);
-            if (tid == 0 && !dead) {
-                if (atomicAdd(&sync[1], 1u) == (uint32_t)p.Q - 1u) {   // the last share of the tile
-                    __threadfence();
-                    sync[0] = 0u;
-                    sync[1] = 0u;
-                    st_release_u32(&sync[2], *(volatile uint32_t *)&hdr->full_steps + 1u);
-                }
-            }
-            SVDC_TRACE_ADD(3, d3);
-        }
-    }
-
-done:
-    SVDC_TRACE_FLUSH(g_trace);
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 1) {
-        tc_fence_after();
-        tmem_dealloc(tmem_base, 512);
-    }
+    if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar, 0u, abort_flag, 99, limit)))
+        record_timeout(p, abort_flag, (uint32_t)(threadIdx.x >> 5), 0u, 0u);
 }
 
 // ------------------------------------------------------------------------- host side ---
@@ -1701,15 +1102,17 @@ int make_map(CUtensorMap *m, const void *base, uint64_t inner, uint64_t rows, ui
     return r == CUDA_SUCCESS ? SVDCACHE_OK : SVDCACHE_ERR_CUDA;
 }
 
+// SMs of the current device (asked every time: a process may drive several devices)
 int num_sms() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        if (n <= 0) n = 148;
-    }
-    return n;
+    int dev = 0, n = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    return n > 0 ? n : 148;
+}
+
+// cudaFuncAttributeMaxDynamicSharedMemorySize is kept per device: set on every call (cheap)
+template <typename K> int allow_big_smem(K kern, size_t bytes) {
+    return record_cuda(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
 }
 
 constexpr size_t kSmemBudget = 227 * 1024;
@@ -1728,7 +1131,6 @@ bool fill_params(const StepArgs &a, UmmaParams &p) {
     {
         const StateLayout SL = state_layout(a.N, a.D, a.k, a.dtype);
         p.chat_off = SL.chat; p.ophi_off = SL.op_hi; p.oplo_off = SL.op_lo;
-        p.chi_off = SL.c_hi; p.clo_off = SL.c_lo; p.sync_off = SL.sync; p.r_off = SL.r;
     }
     p.C_out = a.C_out;
     p.C_stride = a.C_stride;
@@ -1747,11 +1149,10 @@ void fill_groups(const StepArgs &a, UmmaParams &p) {
 }
 
 // Full step: shared memory = A operand region (+ Chat staging when k < 64) | basis ring | F ring | barriers.
-bool fill_full(const StepArgs &a, UmmaParams &p, int cluster = 1) {
+bool fill_full(const StepArgs &a, UmmaParams &p) {
     if (!fill_params(a, p)) return false;
-    p.cluster = cluster;
     fill_groups(a, p);
-    const bool a_tmem = a.k >= 64 && cluster == 1;
+    const bool a_tmem = a.k >= 64;
     // With the operand in TMEM the basis slices may outgrow the 32 KB of fill_groups: wider groups
     // mean fewer, wider MMAs in pass 2 (N = 192 costs ~144 cycles, two of N = 128 ~230) and fewer
     // hand-overs per unit -- as wide as TMEM and, below, shared memory allow (measured: k = 128
@@ -1767,8 +1168,8 @@ bool fill_full(const StepArgs &a, UmmaParams &p, int cluster = 1) {
     // From k = 64 on the A operand lives in tensor memory (the kernel's c_split) and the previous
     // Chat comes through registers: no A region at all, and the shared memory goes to the rings --
     // a third basis slot first (a slice arrives 2000-3000 cycles after its request under load, a
-    // group of MMAs lasts ~1000), a fourth if it costs no F slot.  Below k = 64, and in a cluster,
-    // the operand and the staged Chat share a region of shared memory.
+    // group of MMAs lasts ~1000), a fourth if it costs no F slot.  Below k = 64 the operand and
+    // the staged Chat share a region of shared memory.
     p.chat_stage_off = a_tmem ? 0u : p.a_bytes;
     p.a_region_bytes = a_tmem ? 0u : p.a_bytes + (uint32_t)kTileRows * a.k * 4u;
     p.a_region_bytes = (p.a_region_bytes + 1023u) & ~1023u;
@@ -1791,48 +1192,6 @@ bool fill_full(const StepArgs &a, UmmaParams &p, int cluster = 1) {
 size_t smem_bytes_full(const UmmaParams &p) {
     return 1024 + (size_t)p.a_region_bytes + (size_t)p.v_slots * p.vslice_bytes + (size_t)p.stages * kTileBytes +
            kBarBytes + 64;
-}
-
-// Batched two-phase full step: shared memory = A operand | basis ring | F ring | barriers.
-bool fill_full2(const StepArgs &a, UmmaParams &p) {
-    if (!fill_params(a, p)) return false;
-    fill_groups(a, p);
-    // TMEM: two C accumulators in columns [0, 2k), then at least two stages of the pass-2 ring
-    while (p.gc > 1 && 2 * a.k + 2 * p.gc * kTileCols > 512) --p.gc;
-    if (2 * a.k + 2 * p.gc * kTileCols > 512) return false;
-    p.acc_cols = p.gc * kTileCols;
-    p.acc_stages = (512 - 2 * a.k) / p.acc_cols < kAccStages ? (512 - 2 * a.k) / p.acc_cols : kAccStages;
-    p.vslice_bytes = (uint32_t)p.gc * kTileCols * a.k * 2;
-    const size_t avail = kSmemBudget - 1024 /*alignment*/ - kBar2Bytes - 64;
-    const size_t fixed = (size_t)p.a_bytes + (size_t)p.v_slots * p.vslice_bytes;
-    if (fixed + 4 * (size_t)kTileBytes > avail) return false;
-    p.stages = (int)((avail - fixed) / kTileBytes);
-    if (p.stages > kMaxStages) p.stages = kMaxStages;
-    p.stages &= ~1;
-    // column slices per tile: up to four, as many as there are column groups, and their partial
-    // C's (Q x k floats per row) must fit into the head of an R row (D bf16)
-    const int groups = (p.chunks_total + p.gc - 1) / p.gc;
-    // Column slices per tile, Q in {1, 2, 4, 8}: each slice CTA also combines 128 / Q rows of the
-    // tile, k / Q columns per thread (a multiple of 4).  More slices mean fewer tiles per batch,
-    // and what has to survive in L2 from P1(b) to P2(b) is about four batches' worth of F and R
-    // traffic: Q is the smallest value that keeps one batch of F under ~16 MB.
-    const size_t tile_bytes = (size_t)kTileRows * a.D * 2;
-    p.Q = 1;
-    while (p.Q < 8 && p.Q * 2 <= groups && (a.k / (p.Q * 2)) % 4 == 0 &&
-           (size_t)(num_sms() / p.Q) * tile_bytes > ((size_t)16 << 20))
-        p.Q *= 2;
-    while (p.Q > 1 && (size_t)p.Q * a.k * 4 > (size_t)a.D * 2) p.Q /= 2;
-    if ((size_t)p.Q * a.k * 4 > (size_t)a.D * 2) return false;
-    p.T = p.row_tiles * a.nblocks;
-    p.Bt = num_sms() / p.Q < p.T ? num_sms() / p.Q : p.T;
-    p.nbat = (p.T + p.Bt - 1) / p.Bt;
-    // the chain dump -> all slices there -> combination -> mark -> A operand is some seven memory
-    // round trips long (~10 us under load): with short units it needs two batches to hide behind
-    p.lag = p.Q >= 8 ? 2 : 1;
-    return true;
-}
-size_t smem_bytes_full2(const UmmaParams &p) {
-    return 1024 + (size_t)p.a_bytes + (size_t)p.v_slots * p.vslice_bytes + (size_t)p.stages * kTileBytes + kBar2Bytes + 64;
 }
 
 bool fill_cached(const StepArgs &a, UmmaParams &p) {
@@ -1889,13 +1248,14 @@ int umma_cached_step(const StepArgs &a, cudaStream_t s) {
     // whole tiles).  With a single operand buffer (k >= 128) every unit waits for its own copy of
     // the tile's A operand with empty rings (~4 chunks' worth, plus the a_bytes it re-reads), which
     // outweighs that: 5.7 TB/s with whole tiles at k = 128, 4.2 with single-group units.
+    const int sms = num_sms();
     const int tiles = p.row_tiles * a.nblocks;
     const int groups_total = (p.chunks_total + p.gc - 1) / p.gc;
     const int unit_cost = p.a_bufs == 1 ? (int)((p.a_bytes + 2 * kTileBytes - 1) / (2 * kTileBytes)) + 4 : 0;
     auto load_of = [&](int ds, int *eff_out, int *gps_out) {
         const int gps = (groups_total + ds - 1) / ds;            // groups per slice
         const int eff = (groups_total + gps - 1) / gps;          // slices that result
-        const int rounds = (tiles * eff + num_sms() - 1) / num_sms();
+        const int rounds = (tiles * eff + sms - 1) / sms;
         *eff_out = eff; *gps_out = gps;
         return rounds * (gps * p.gc + unit_cost);
     };
@@ -1933,118 +1293,29 @@ int umma_cached_step(const StepArgs &a, cudaStream_t s) {
     if (rc) return rc;
 
     const size_t smem = smem_bytes_cached(p);
-    static bool attr_set = false;
-    if (!attr_set) {
-        rc = record_cuda(cudaFuncSetAttribute(umma_cached_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              (int)kSmemBudget));
-        if (rc) return rc;
-        attr_set = true;
-    }
-    const int grid = p.units < num_sms() ? p.units : num_sms();
+    rc = allow_big_smem(umma_cached_kernel, kSmemBudget);
+    if (rc) return rc;
+    const int grid = p.units < sms ? p.units : sms;
     umma_cached_kernel<<<grid, kThreadsCached, smem, s>>>(tm_r, tm_v, tm_ahi, tm_alo, tm_out, p);
     count_launch();
     return check_last_launch();
 }
 
-// Largest number of 2-CTA clusters of the full-step kernel that can be resident at once.
-int max_full_clusters(size_t smem) {
-    static int cached = -1;
-    if (cached >= 0) return cached;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(2 * num_sms());
-    cfg.blockDim = dim3(kThreadsFull);
-    cfg.dynamicSmemBytes = smem;
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
-    int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, umma_full_kernel<true, false>, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
-    cached = n;
-    return n;
-}
-
-// Batched two-phase schedule; returns SVDCACHE_ERR_BAD_SHAPE when the shape is outside it.
-int umma_full2_step(const StepArgs &a, cudaStream_t s) {
+int umma_wait_selftest(void *state, long long limit_cycles, cudaStream_t s) {
     UmmaParams p{};
-    if (!fill_full2(a, p)) return SVDCACHE_ERR_BAD_SHAPE;
-    const StateLayout SL = state_layout(a.N, a.D, a.k, a.dtype);
-    const BasisLayout BL = basis_layout(a.D, a.k, a.dtype);
-    CUtensorMap tm_f, tm_vt, tm_v, tm_rout, tm_chi, tm_clo;
-    int rc = make_map(&tm_f, a.F, a.D, a.N, a.nblocks, (uint64_t)a.ld * 2, a.F_stride, kTileCols, kTileRows);
-    if (rc) return rc;
-    rc = make_map(&tm_vt, (const char *)a.basis + BL.vt_bf16, a.D, a.k, a.nblocks, (uint64_t)a.D * 2,
-                  a.basis_stride, kTileCols, a.k);
-    if (rc) return rc;
-    rc = make_map(&tm_v, (const char *)a.basis + BL.v_bf16, a.k, a.D, a.nblocks, (uint64_t)a.k * 2, a.basis_stride,
-                  p.kb_elems, p.gc * kTileCols);
-    if (rc) return rc;
-    rc = make_map(&tm_rout, (char *)a.state + SL.r, a.D, a.N, a.nblocks, (uint64_t)a.D * 2, a.state_stride,
-                  kTileCols, kSlabRows);
-    if (rc) return rc;
-    rc = make_map(&tm_chi, (char *)a.state + SL.c_hi, a.k, a.N, a.nblocks, (uint64_t)a.k * 2, a.state_stride,
-                  p.kb_elems, kTileRows);
-    if (rc) return rc;
-    rc = make_map(&tm_clo, (char *)a.state + SL.c_lo, a.k, a.N, a.nblocks, (uint64_t)a.k * 2, a.state_stride,
-                  p.kb_elems, kTileRows);
-    if (rc) return rc;
-    static bool attr_set = false;
-    if (!attr_set) {
-        rc = record_cuda(cudaFuncSetAttribute(umma_full2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              (int)kSmemBudget));
-        if (rc) return rc;
-        attr_set = true;
-    }
-    // every CTA of the grid must be resident at once (CTAs wait for marks that other CTAs set):
-    // one CTA per SM, at most as many CTAs as SMs
-    umma_full2_kernel<<<p.Bt * p.Q, kThreadsFull2, smem_bytes_full2(p), s>>>(tm_f, tm_vt, tm_v, tm_rout, tm_chi, tm_clo, p);
+    p.state = (char *)state;
+    p.nblocks = 1;
+    wait_selftest_kernel<<<1, 64, 0, s>>>(p, limit_cycles);
     count_launch();
     return check_last_launch();
 }
 
 int umma_full_step(const StepArgs &a, cudaStream_t s) {
-    if (a.cluster_split == 2) {   // batched two-phase schedule requested
-        const int rc2 = umma_full2_step(a, s);
-        if (rc2 != SVDCACHE_ERR_BAD_SHAPE) return rc2;
-    }
     UmmaParams p{};
     if (!fill_full(a, p)) return SVDCACHE_ERR_BAD_SHAPE;
     p.dsplit = 1;
     p.chunks_per_slice = p.chunks_total;
     p.units = p.row_tiles * a.nblocks;
-
-    static bool attr_set = false;
-    if (!attr_set) {
-        int rc0 = record_cuda(cudaFuncSetAttribute(umma_full_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   (int)kSmemBudget));
-        if (rc0) return rc0;
-        rc0 = record_cuda(cudaFuncSetAttribute(umma_full_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               (int)kSmemBudget));
-        if (rc0) return rc0;
-        rc0 = record_cuda(cudaFuncSetAttribute(umma_full_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               (int)kSmemBudget));
-        if (rc0) return rc0;
-        attr_set = true;
-    }
-    // Two CTAs per row tile (each streams half the columns in both passes) halve the F bytes
-    // that must survive in L2 between the passes.  On request only: the exchange of the partial
-    // C's lengthens the serial part of every tile and the F ring is shorter, which today costs
-    // more than the L2 hits bring.  Needs the split operand layout (k >= 64), at least two
-    // column groups and an F ring of six slots.
-    int nclusters = 0;
-    {
-        UmmaParams pc{};
-        const int groups = (p.chunks_total + p.gc - 1) / p.gc;
-        if (a.cluster_split == 1 && a.k >= 64 && groups >= 2 && fill_full(a, pc, 2) && pc.stages >= 6) {
-            const int fit = max_full_clusters(smem_bytes_full(pc));
-            if (fit >= num_sms() / 2 - 4) {   // else the cluster placement leaves too many SMs idle
-                pc.dsplit = 1; pc.chunks_per_slice = pc.chunks_total; pc.units = p.units;
-                p = pc;
-                nclusters = p.units < fit ? p.units : fit;
-            }
-        }
-    }
 
     const StateLayout SL = state_layout(a.N, a.D, a.k, a.dtype);
     const BasisLayout BL = basis_layout(a.D, a.k, a.dtype);
@@ -2065,26 +1336,17 @@ int umma_full_step(const StepArgs &a, cudaStream_t s) {
     if (rc) return rc;
 
     const size_t smem = smem_bytes_full(p);
-    if (p.cluster == 2) {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(2 * nclusters);
-        cfg.blockDim = dim3(kThreadsFull);
-        cfg.dynamicSmemBytes = smem;
-        cfg.stream = s;
-        cudaLaunchAttribute attr;
-        attr.id = cudaLaunchAttributeClusterDimension;
-        attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
-        cfg.attrs = &attr;
-        cfg.numAttrs = 1;
-        rc = record_cuda(cudaLaunchKernelEx(&cfg, umma_full_kernel<true, false>, tm_f, tm_vt, tm_v, tm_rout, tm_chat, p));
-        count_launch();
-        return rc ? rc : check_last_launch();
+    const int sms = num_sms();
+    const int grid = p.units < sms ? p.units : sms;
+    if (a.k >= 64) {   // operand in tensor memory (fill_full has sized the rings for it)
+        rc = allow_big_smem(umma_full_kernel<true>, kSmemBudget);
+        if (rc) return rc;
+        umma_full_kernel<true><<<grid, kThreadsFull, smem, s>>>(tm_f, tm_vt, tm_v, tm_rout, tm_chat, p);
+    } else {
+        rc = allow_big_smem(umma_full_kernel<false>, kSmemBudget);
+        if (rc) return rc;
+        umma_full_kernel<false><<<grid, kThreadsFull, smem, s>>>(tm_f, tm_vt, tm_v, tm_rout, tm_chat, p);
     }
-    const int grid = p.units < num_sms() ? p.units : num_sms();
-    if (a.k >= 64)   // operand in tensor memory (fill_full has sized the rings for it)
-        umma_full_kernel<false, true><<<grid, kThreadsFull, smem, s>>>(tm_f, tm_vt, tm_v, tm_rout, tm_chat, p);
-    else
-        umma_full_kernel<false, false><<<grid, kThreadsFull, smem, s>>>(tm_f, tm_vt, tm_v, tm_rout, tm_chat, p);
     count_launch();
     return check_last_launch();
 }

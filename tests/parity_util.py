@@ -11,7 +11,8 @@ from paper_2601_07396_b200 import binding as sc
 
 # Tolerances of the comparison with the fp64 oracle, per output array (C, Chat, R, Fhat):
 #   fp32 I/O: relative Frobenius error <= 1e-5
-#   bf16 I/O: relative Frobenius error <= 5e-3 and max-abs error <= 2e-2 * rms(F)
+#   bf16 I/O: relative Frobenius error <= 5e-3 and max-abs error <= 2e-2 * rms(F) (one bf16 ulp of
+#             the reference value where that is larger: see check_close)
 TOL = {sc.F32: dict(rel=1e-5, maxabs=None), sc.BF16: dict(rel=5e-3, maxabs=2e-2)}
 
 
@@ -21,18 +22,30 @@ def rel_fro(x: np.ndarray, ref: np.ndarray) -> float:
     return float(num / den) if den > 0 else float(num)
 
 
-def check_close(name, got, ref, dtype, rms_f, coeff=False):
-    """Assert `got` (torch tensor or ndarray) against the oracle's `ref`."""
+def check_close(name, got, ref, dtype, rms_f, coeff=0):
+    """Assert `got` (torch tensor or ndarray) against the oracle's `ref`; `coeff` = D for the
+    fp32 coefficient arrays (see below), 0 for arrays in the I/O dtype."""
     if isinstance(got, torch.Tensor):
         got = got.detach().double().cpu().numpy()
     tol = TOL[dtype]
     rel = rel_fro(got, ref)
-    # coefficient arrays are fp32 in both modes and are not rounded to bf16
-    bound = 1e-5 if (coeff and dtype == sc.F32) else tol["rel"]
+    # Coefficient arrays (C, Chat) are fp32 in both modes and never rounded to bf16.  `coeff` is
+    # the width D they were reduced over: bf16 products are exact in fp32, and the tensor cores
+    # truncate the fp32 running sum once per 16 columns, a one-sided error of at most
+    # 2^-24 * D / 4 = 4e-9 * D relative (D = 1024: 1.3e-6 measured; D = 8192: 1.8e-5), so the
+    # bound is the fp32 one up to D = 2500 and 4e-9 * D beyond; fp32 I/O accumulates in fp64.
+    bound = (1e-5 if dtype == sc.F32 else max(1e-5, 4e-9 * float(coeff))) if coeff else tol["rel"]
     assert rel <= bound, f"{name}: relative Frobenius error {rel:.3e} > {bound:.1e}"
     if tol["maxabs"] is not None:
-        mx = float(np.abs(got - ref).max())
-        assert mx <= tol["maxabs"] * rms_f, f"{name}: max-abs error {mx:.3e} > {tol['maxabs']}*rms(F)={tol['maxabs'] * rms_f:.3e}"
+        # Element-wise bound of the bf16 mode: 2e-2 * rms(F) -- or one bf16 ulp of the reference
+        # value where that is larger.  An output stored in bf16 is off by up to half an ulp
+        # (2^-9 |x|) however it was computed, which passes 2e-2 * rms(F) once |x| > 10 rms(F);
+        # among the 1e8 elements sampled at the full FLUX size a few are that large.
+        err = np.abs(got - ref)
+        bound_el = np.maximum(tol["maxabs"] * rms_f, 2.0 ** -8 * np.abs(ref))
+        worst = int(np.argmax(err - bound_el))
+        assert (err <= bound_el).all(), (f"{name}: element error {err.flat[worst]:.3e} > "
+                                        f"max({tol['maxabs']}*rms(F)={tol['maxabs'] * rms_f:.3e}, 2^-8*|ref|={2.0 ** -8 * abs(ref.flat[worst]):.3e})")
     return rel
 
 

@@ -77,29 +77,84 @@ def test_flux_width_calibration_single_snapshot():
     _compare(stack, spec.k, Vk, lam, tr)
 
 
-def test_flux_stack_of_73728_rows_against_an_fp64_product():
-    """The tensor-core Gram at a size the CPU oracle would need minutes for: 16 snapshots of
-    the FLUX-shaped stream (73,728 x 3072, bf16, k = 64).  The reference is the definition
-    evaluated with library routines in fp64 on the same device data (G = F^T F, then a full
-    symmetric eigen-decomposition); the eigen-gap at k of this spectrum is only a few 1e-6 of
-    lambda_1, so this is where an fp32 sum over the whole stack would lose the subspace."""
+def _compare_large(stack: torch.Tensor, k: int, Vk, lam, tr, min_gap=1e-7):
+    """The same comparison for stacks whose fp64 copy would not fit comfortably on the host: the
+    oracle's Gram routine is called snapshot by snapshot (the sum of the partial Gram matrices is
+    the definition, Eq. 4), then the oracle's eigen-solver on the total."""
+    M, D = stack.shape
+    G = np.zeros((D, D))
+    for lo in range(0, M, 4608):
+        G += oracle.gram(stack[lo:lo + 4608].double().cpu().numpy())
+    w, Z = oracle.eigh_desc(G)
+    V = Vk.double().cpu().numpy()
+    gap = (w[k - 1] - w[k]) / w[0]
+    assert gap > min_gap, f"eigen-gap at k too small to grade angles: {gap:.2e}"
+    cos = np.linalg.svd(Z[:, :k].T @ V, compute_uv=False)
+    assert cos.min() >= COS_MIN, f"smallest principal-angle cosine {cos.min():.8f} (gap {gap:.2e})"
+    # eigenvalues and trace on the tensor-core path: see _compare
+    np.testing.assert_allclose(lam.cpu().numpy(), w[:k], rtol=2e-5, atol=5e-6 * w[0])
+    assert float(tr.cpu()[0]) == pytest.approx(float(np.trace(G)), rel=2e-5)
+    np.testing.assert_allclose(V.T @ V, np.eye(k), atol=5e-6)
+    return cos.min(), gap
+
+
+def test_flux_stack_of_73728_rows():
+    """The middle stack of the calibration sweep: 16 snapshots of the FLUX-shaped stream
+    (73,728 x 3072, bf16, k = 64) against the oracle.  The eigen-gap at k of this spectrum is only
+    a few 1e-6 of lambda_1, so this is where an fp32 sum over the whole stack would lose the
+    subspace."""
     spec = streams.FLUX
     stack = streams.calibration_stack(spec, 0, device=DEV, trajectories=(1, 2), timesteps=spec.calib_timesteps)
     assert stack.shape == (73728, 3072)
-    k = spec.k
-    Vk, lam, tr, info = sc.svdcache_calibrate(stack, k)
-    G = torch.zeros(3072, 3072, dtype=torch.float64, device=DEV)
-    for lo in range(0, stack.shape[0], 8192):
-        blk = stack[lo:lo + 8192].double()
-        G += blk.t() @ blk
-    w, Q = torch.linalg.eigh(G)
-    w, Q = w.flip(0), Q.flip(1)
-    gap = float((w[k - 1] - w[k]) / w[0])
-    assert gap > 1e-7, gap
-    cos = torch.linalg.svdvals(Q[:, :k].t() @ Vk.double())
-    assert float(cos.min()) >= COS_MIN, f"smallest principal-angle cosine {float(cos.min()):.8f} (gap {gap:.2e})"
-    np.testing.assert_allclose(lam.cpu().numpy(), w[:k].cpu().numpy(), rtol=2e-5, atol=5e-6 * float(w[0]))
-    assert float(tr.cpu()[0]) == pytest.approx(float(torch.trace(G)), rel=2e-5)
+    Vk, lam, tr, info = sc.svdcache_calibrate(stack, spec.k)
+    _compare_large(stack, spec.k, Vk, lam, tr)
+
+
+def test_flux_configured_stack_of_294912_rows():
+    """The FLUX configuration's own calibration stack: 8 trajectories x 8 timesteps x 4608 rows =
+    294,912 x 3072 (the stack the calibration timing is quoted on), against the oracle."""
+    spec = streams.FLUX
+    stack = streams.calibration_stack(spec, 5, device=DEV)
+    assert stack.shape == (294912, 3072)
+    Vk, lam, tr, info = sc.svdcache_calibrate(stack, spec.k)
+    _compare_large(stack, spec.k, Vk, lam, tr)
+
+
+def test_hunyuan_configuration_rank_and_width():
+    """The HunyuanVideo configuration's calibration: k = 128 at D = 3072 (the Ritz problem of 160
+    columns no longer fits shared memory and runs its Jacobi sweeps from global memory), on two
+    snapshots of 8192 rows, which takes the tensor-core Gram."""
+    spec = streams.HUNYUAN
+    stack = streams.calibration_stack(spec, 2, device=DEV, rows_per_snapshot=8192)
+    assert stack.shape == (16384, 3072) and stack.dtype == torch.bfloat16
+    Vk, lam, tr, info = sc.svdcache_calibrate(stack, spec.k)
+    _compare_large(stack, spec.k, Vk, lam, tr)
+
+
+def test_finish_refuses_a_workspace_begun_for_another_shape():
+    """svdcache_calibrate_finish (and _accumulate) against what svdcache_calibrate_begin laid out."""
+    L = sc.lib()
+    p = lambda t: ctypes.c_void_p(t.data_ptr())
+    s = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    ws = torch.empty(sc.svdcache_calibrate_workspace_bytes(512, 64), dtype=torch.uint8, device=DEV)
+    spec = streams.StreamSpec("cal", blocks=1, rows=300, D=256, dtype="f32", k=8, T=2, interval=1,
+                              rank=48, amp=40.0, power=1.0, noise_std=0.02)
+    F = streams.BlockStream(spec, 0, device=DEV).features(1)
+    Vk = torch.empty(512, 64, device=DEV)
+    sc.svdcache_calibrate_begin(256, 16, ws)
+    sc.svdcache_calibrate_accumulate(F, ws)
+    # another width, and a larger rank than the workspace was begun for
+    assert L.svdcache_calibrate_finish(512, 16, p(Vk), None, None, None, p(ws), ws.numel(), s) == -5
+    assert L.svdcache_calibrate_finish(256, 32, p(Vk), None, None, None, p(ws), ws.numel(), s) == -5
+    # a chunk of another width poisons the accumulation
+    F2 = torch.randn(300, 128, device=DEV)
+    assert L.svdcache_calibrate_accumulate(p(F2), 300, 128, 128, 0, p(ws), ws.numel(), s) == 0
+    assert L.svdcache_calibrate_finish(256, 16, p(Vk), None, None, None, p(ws), ws.numel(), s) == -5
+    # begun again, the same workspace works, also for a smaller rank than begun
+    sc.svdcache_calibrate_begin(256, 16, ws)
+    sc.svdcache_calibrate_accumulate(F, ws)
+    V8, lam, tr, info = sc.svdcache_calibrate_finish(256, 8, ws, strict=False)
+    _compare(F, 8, V8, lam, tr)
 
 
 @pytest.mark.parametrize("M,D,k,dtype", [(100, 64, 8, "f32"), (1000, 264, 24, "bf16"), (37, 128, 16, "f32"),
