@@ -35,12 +35,14 @@ METRIC = "fused full/cached-step HBM GB/s and % of B200 HBM roofline (FLUX-shape
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel (the batched cached
-# step, tcgen05 family), per block, from the ncu capture summarised in
-# profiles/umma_cached_kernel_flux_8blocks.txt: taken on 8 blocks of the same shape and
-# scaled by the block count (traffic is proportional to the blocks a launch covers).  The
-# tail of the output that is still in L2 when the kernel ends is not in the counter.
-NCU_TRAFFIC_BYTES_PER_BLOCK = {("flux", 2): 52100928}
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the timed kernels, from ncu
+# captures of this very launch shape (all blocks of the workload in one batched launch; the
+# summaries under profiles/ name the commands).  Keyed by (workload, blocks, kernel family);
+# any other shape reports null -- nothing is scaled.
+NCU_TRAFFIC_BYTES = {
+    "cached": {},
+    "full": {},
+}
 
 
 def algorithmic_bytes(spec: streams.StreamSpec, nblocks: int):
@@ -180,6 +182,140 @@ def build_workload(spec, nblocks, device, block_offset=0, calibrate_rows=None):
     return dict(F=F, bases=bases, state=state, Fhat=Fhat, dt=dt, cal_ms=cal_ms, cal_rows=n_cal)
 
 
+def measure_steps(sc, spec, wl, steps, warmup, barrier, sampler=None):
+    """`warmup` untimed steps, then `steps` timed ones (one step = one batched full step + interval-1
+    batched cached steps over all blocks of `wl`), CUDA events on the launching stream around the
+    whole region and around every launch."""
+    F, bases, state, Fhat = wl["F"], wl["bases"], wl["state"], wl["Fhat"]
+    k, beta, interval = spec.k, spec.beta, spec.interval
+
+    def one_step(events=None):
+        if events is not None:
+            e = torch.cuda.Event(enable_timing=True); e.record(); events.append(e)
+        sc.svdcache_full_step_batched(F, bases, state, k, beta)
+        if events is not None:
+            e = torch.cuda.Event(enable_timing=True); e.record(); events.append(e)
+        for j in range(1, interval):
+            sc.svdcache_cached_step_batched(state, bases, Fhat, k, steps_since_full=j)
+            if events is not None:
+                e = torch.cuda.Event(enable_timing=True); e.record(); events.append(e)
+
+    for _ in range(warmup):
+        one_step()
+    barrier()
+    if sampler is not None:
+        sampler.start()
+        time.sleep(0.25)
+    launches0 = sc.svdcache_kernel_launches()
+    events = []
+    t_host0 = time.time()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(steps):
+        one_step(events)
+    stop.record()
+    barrier()
+    t_host1 = time.time()
+    clocks = sampler.stop(t_host0, t_host1) if sampler is not None else None
+    launches = sc.svdcache_kernel_launches() - launches0
+    per = interval + 1
+    full_ms, cached_ms = [], []
+    for s_ in range(steps):
+        ev = events[s_ * per:(s_ + 1) * per]
+        full_ms.append(ev[0].elapsed_time(ev[1]))
+        for j in range(1, interval):
+            cached_ms.append(ev[j].elapsed_time(ev[j + 1]))
+    return dict(total_ms=start.elapsed_time(stop), full_ms=full_ms, cached_ms=cached_ms, launches=launches, clocks=clocks)
+
+
+def parity_of_timed_buffers(sc, spec, wl, rows_per_block=256):
+    """Outside the timed region: the state and Fhat the timed launches left behind, sampled rows of
+    the first, the middle and the last block, against the fp64 oracle driven through as many full
+    steps (of the same F) as the state has seen.  Returns the worst relative Frobenius errors and
+    raises SystemExit when a bound of the parity tests is exceeded."""
+    from oracle import svdcache_oracle as oracle
+    import numpy as np
+    F, bases, state, Fhat, dt = wl["F"], wl["bases"], wl["state"], wl["Fhat"], wl["dt"]
+    nb, N, D = F.shape
+    k = spec.k
+    beta = float(np.float32(spec.beta))
+    rows = streams.sample_rows(N, rows_per_block, tile=128)
+    rows_d = rows.to(F.device)
+    worst = {"Chat": 0.0, "R": 0.0, "Fhat": 0.0}
+    checked = sorted({0, nb // 2, nb - 1})
+    steps_seen = 0
+    for b in checked:
+        steps_seen, status = sc.svdcache_state_query(state[b])
+        if status != 0 or steps_seen < 1:
+            raise SystemExit(f"bench parity: block {b} has status {status} after {steps_seen} full steps")
+        V = (sc.basis_views(bases[b], D, k, dt)[0 if dt == sc.F32 else 2]).double().cpu().numpy()
+        Fh = F[b][rows_d].double().cpu().numpy()
+        chat = None
+        for _ in range(int(steps_seen)):
+            C, R, chat = oracle.full_step(Fh, V, beta, chat)
+        ref = oracle.cached_step(chat, V, R)
+        chat_v, r_v = sc.state_views(state[b], N, D, k, dt)
+        for name, got, want in (("Chat", chat_v[rows_d], chat), ("R", r_v[rows_d], R), ("Fhat", Fhat[b][rows_d], ref)):
+            g = got.double().cpu().numpy()
+            err = float(np.linalg.norm(g - want) / np.linalg.norm(want))
+            worst[name] = max(worst[name], err)
+    io_bound = 1e-5 if dt == sc.F32 else 5e-3
+    chat_bound = 1e-5 if dt == sc.F32 else max(1e-5, 4e-9 * D)
+    bounds = {"Chat": chat_bound, "R": io_bound, "Fhat": io_bound}
+    bad = {n_: e for n_, e in worst.items() if not e <= bounds[n_]}
+    if bad:
+        raise SystemExit(f"bench parity failed: {bad} against {bounds}")
+    return {"rows": int(len(rows)) * len(checked), "blocks": checked, "full_steps_replayed": int(steps_seen),
+            "Chat": worst["Chat"], "R": worst["R"], "Fhat": worst["Fhat"], "bounds": bounds,
+            "against": "fp64 oracle on sampled rows of the buffers the timed launches wrote"}
+
+
+def roofline_objects(spec, nblocks, full_ms, cached_ms, peak, peak_kind, path_used):
+    b_full, b_cached = algorithmic_bytes(spec, nblocks)
+    c_ms = sum(cached_ms) / max(1, len(cached_ms))
+    f_ms = sum(full_ms) / max(1, len(full_ms))
+    c_gbs = b_cached / (c_ms * 1e-3) / 1e9 if cached_ms else None
+    f_gbs = b_full / (f_ms * 1e-3) / 1e9
+    roof = {"bound": "hbm", "kernel": "cached step (batched)",
+            "achieved": round(c_gbs, 2) if c_gbs else None, "peak": peak,
+            "peak_source": f"{peak_kind} copy bandwidth", "unit": "GB/s",
+            "frac": round(c_gbs / peak, 4) if c_gbs else None,
+            "frac_of_nominal_8TBs": round(c_gbs / NOMINAL_HBM_GBS, 4) if c_gbs else None,
+            "traffic": NCU_TRAFFIC_BYTES["cached"].get((spec.name, nblocks, path_used)),
+            "algorithmic_bytes": b_cached, "avg_launch_ms": round(c_ms, 4)}
+    roof_full = {"bound": "hbm", "kernel": "full step (batched)", "achieved": round(f_gbs, 2),
+                 "peak": peak, "unit": "GB/s", "frac": round(f_gbs / peak, 4),
+                 "frac_of_nominal_8TBs": round(f_gbs / NOMINAL_HBM_GBS, 4),
+                 "traffic": NCU_TRAFFIC_BYTES["full"].get((spec.name, nblocks, path_used)),
+                 "algorithmic_bytes": b_full, "avg_launch_ms": round(f_ms, 4)}
+    return roof, roof_full
+
+
+def hunyuan_addendum(sc, args, device, peak, peak_kind):
+    """The same two kernels on the HunyuanVideo-shaped stream (N = 118,800 rows, k = 128): 8 of its
+    60 blocks resident at a time (about 19 GB with state; every launch streams > 11 GB), fewer
+    steps.  The headline value stays the FLUX-shaped one."""
+    spec = streams.SPECS["hunyuan"]
+    nblocks = 8
+    wl = build_workload(spec, nblocks, device)
+    steps = max(3, min(args.steps, 6))
+    m = measure_steps(sc, spec, wl, steps, 3, torch.cuda.synchronize)
+    path_used = sc.svdcache_last_path()
+    roof, roof_full = roofline_objects(spec, nblocks, m["full_ms"], m["cached_ms"], peak, peak_kind, path_used)
+    b_full, b_cached = algorithmic_bytes(spec, nblocks)
+    step_bytes = b_full + (spec.interval - 1) * b_cached
+    out = {"config": {"workload": "hunyuan-shaped stream", "blocks": nblocks, "rows": spec.rows, "D": spec.D,
+                      "k": spec.k, "interval": spec.interval, "steps": steps, "warmup": 3},
+           "value": round(step_bytes * steps / (m["total_ms"] * 1e-3) / 1e9, 2), "unit": "GB/s",
+           "ms_per_step": round(m["total_ms"] / steps, 4),
+           "roofline": roof, "roofline_full_step": roof_full,
+           "tokens_blocks_per_s": round(spec.rows * nblocks * spec.interval * steps / (m["total_ms"] * 1e-3), 1),
+           "gpu_launches": int(m["launches"])}
+    if not args.no_parity:
+        out["parity"] = parity_of_timed_buffers(sc, spec, wl)
+    return out
+
+
 def run_ours(args):
     from paper_2601_07396_b200 import binding as sc
     rank, world, local = dist_env()
@@ -201,51 +337,18 @@ def run_ours(args):
     bytes_full, bytes_cached = algorithmic_bytes(spec, nblocks)
     step_bytes = bytes_full + (interval - 1) * bytes_cached
 
-    def one_step(events=None):
-        if events is not None:
-            e = torch.cuda.Event(enable_timing=True); e.record(); events.append(e)
-        sc.svdcache_full_step_batched(F, bases, state, k, beta)
-        if events is not None:
-            e = torch.cuda.Event(enable_timing=True); e.record(); events.append(e)
-        for j in range(1, interval):
-            sc.svdcache_cached_step_batched(state, bases, Fhat, k, steps_since_full=j)
-            if events is not None:
-                e = torch.cuda.Event(enable_timing=True); e.record(); events.append(e)
-
     def barrier():
         if world > 1:
             import torch.distributed as dist
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
-        one_step()
-    barrier()
-
     # ---- device-resident timing: K steps, CUDA events on the launching stream ----
     sampler = ClockSampler(local)
-    sampler.start()
-    time.sleep(0.25)
-    launches0 = sc.svdcache_kernel_launches()
-    events = []
-    t_host0 = time.time()
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    start.record()
-    for _ in range(args.steps):
-        one_step(events)
-    stop.record()
-    barrier()
-    t_host1 = time.time()
-    clocks = sampler.stop(t_host0, t_host1)
-    launches = sc.svdcache_kernel_launches() - launches0
-    total_ms = reduce_max(start.elapsed_time(stop), world, device)
-    per = interval + 1
-    full_ms, cached_ms = [], []
-    for s in range(args.steps):
-        ev = events[s * per:(s + 1) * per]
-        full_ms.append(ev[0].elapsed_time(ev[1]))
-        for j in range(1, interval):
-            cached_ms.append(ev[j].elapsed_time(ev[j + 1]))
+    m = measure_steps(sc, spec, wl, args.steps, args.warmup, barrier, sampler)
+    clocks, launches = m["clocks"], m["launches"]
+    total_ms = reduce_max(m["total_ms"], world, device)
+    full_ms, cached_ms = m["full_ms"], m["cached_ms"]
     path_used = sc.svdcache_last_path()
 
     # ---- end to end: host buffers, H2D of F and D2H of the final Fhat every step ----
@@ -289,11 +392,7 @@ def run_ours(args):
     peak, peak_kind = measured_peak()
     value = whole_job_value(step_bytes, args.steps, world, total_ms)
     e2e_value = whole_job_value(step_bytes, e2e_steps, world, e2e_ms)
-    cached_avg_ms = sum(cached_ms) / max(1, len(cached_ms))
-    full_avg_ms = sum(full_ms) / max(1, len(full_ms))
-    cached_gbs = bytes_cached / (cached_avg_ms * 1e-3) / 1e9 if cached_ms else None
-    full_gbs = bytes_full / (full_avg_ms * 1e-3) / 1e9
-    traffic = NCU_TRAFFIC_BYTES_PER_BLOCK.get((spec.name, path_used))
+    roof, roof_full = roofline_objects(spec, nblocks, full_ms, cached_ms, peak, peak_kind, path_used)
     line = {
         "metric": METRIC, "value": round(value, 2), "unit": "GB/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(total_ms / args.steps, 4),
@@ -305,18 +404,10 @@ def run_ours(args):
                    "l2": "inputs larger than L2 (each launch streams >= 1 GB)" if step_bytes > 6e8 else
                          "inputs smaller than L2: launch-bound parity config, not a roofline config",
                    "kernel_family": {1: "cuda-core", 2: "tcgen05"}.get(path_used, "?"),
+                   "library": sc.LIB_PATH,
                    "parallelism": f"blocks replicated per rank x{world}, no collective"},
-        "roofline": {"bound": "hbm", "kernel": "cached step (batched)",
-                     "achieved": round(cached_gbs, 2) if cached_gbs else None, "peak": peak,
-                     "peak_source": f"{peak_kind} copy bandwidth", "unit": "GB/s",
-                     "frac": round(cached_gbs / peak, 4) if cached_gbs else None,
-                     "frac_of_nominal_8TBs": round(cached_gbs / NOMINAL_HBM_GBS, 4) if cached_gbs else None,
-                     "traffic": traffic * nblocks if traffic else None,
-                     "algorithmic_bytes": bytes_cached, "avg_launch_ms": round(cached_avg_ms, 4)},
-        "roofline_full_step": {"bound": "hbm", "kernel": "full step (batched)", "achieved": round(full_gbs, 2),
-                               "peak": peak, "unit": "GB/s", "frac": round(full_gbs / peak, 4),
-                               "frac_of_nominal_8TBs": round(full_gbs / NOMINAL_HBM_GBS, 4),
-                               "algorithmic_bytes": bytes_full, "avg_launch_ms": round(full_avg_ms, 4)},
+        "roofline": roof,
+        "roofline_full_step": roof_full,
         "tokens_blocks_per_s": round(world * spec.rows * nblocks * interval * args.steps / (total_ms * 1e-3), 1),
         "e2e": {"value": round(e2e_value, 2), "unit": "GB/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps,
@@ -326,8 +417,14 @@ def run_ours(args):
         "calibration": {"rows": wl["cal_rows"], "median_ms_per_block": round(statistics.median(wl["cal_ms"]), 3),
                         "note": "one-off per block, outside the timed steps"},
     }
+    if not args.no_parity:
+        line["parity"] = parity_of_timed_buffers(sc, spec, wl)
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(spec, F, bases, dt, budget_s=args.cpu_seconds)
+    if world == 1 and spec.name == "flux" and not args.blocks and not args.no_hunyuan:
+        del F, bases, state, Fhat, F_host, out_host, wl
+        torch.cuda.empty_cache()
+        line["hunyuan"] = hunyuan_addendum(sc, args, device, peak, peak_kind)
     print(json.dumps(line), flush=True)
     if world > 1:
         import torch.distributed as dist
@@ -510,6 +607,8 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--ref-rows", type=int, default=1024)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-parity", action="store_true", help="skip the oracle check of the timed buffers")
+    ap.add_argument("--no-hunyuan", action="store_true", help="skip the HunyuanVideo-shaped addendum of the default run")
     ap.add_argument("--calib-rows", type=int, default=0, help="rows of the per-block calibration stack (default: min(N, 4608))")
     ap.add_argument("--sweep", action="store_true", help="rank and calibration sweep on the FLUX shape")
     args = ap.parse_args()

@@ -18,7 +18,12 @@
  * Pins (tests/test_oracle_*.py): orthonormality, trace and Eckart-Young identities,
  * one-sided Jacobi SVD on small matrices, numpy's eigh/svd on the same inputs,
  * exact reconstruction at k = D, residual orthogonality, the energy split
- * |F|^2 = |C|^2 + |R|^2, EMA closed forms, and hand-computed fixtures.
+ * |F|^2 = |C|^2 + |R|^2, EMA closed forms, and hand-computed fixtures; for the routines beyond
+ * the method itself (tests/test_oracle_extensions.py): the residual EMA against its closed
+ * forms and against oracle_full_step at beta_r = 0, the forecasts against polynomial sequences
+ * (exactness of the Newton form, the known lag of the Taylor form), numpy's polynomial fit, and
+ * hand-computed values; the left factors against U diag(sigma) V^T = F_k and U^T U = I on the
+ * calibration stack itself.
  */
 #include <math.h>
 #include <stdint.h>
@@ -347,6 +352,83 @@ void oracle_cached_step(const double *Chat, const double *Vk, const double *R, i
             fh[d] = s + r[d];
         }
     }
+}
+
+/* ------------------------------------------------------------------------------------
+ * Full step with a smoothed residual (the ablation of Sec. 4.5, Fig. 4(c): "EMA on both").
+ * As oracle_full_step, except that the stored residual is itself an EMA of the residuals of
+ * the full steps:
+ *   rhat = r                                  on the first full step
+ *        = beta_r rhat + (1 - beta_r) r       afterwards          (r = f - V_k c, Eq. 10)
+ * beta_r = 0 is the method itself (Sec. 3.5: the residual is reused as it is); beta = 0
+ * together with beta_r = 0 is "reuse on both" (Eq. 3).  Rhat (N x D) is updated in place.
+ * ---------------------------------------------------------------------------------- */
+void oracle_full_step_residual_ema(const double *F, int64_t N, int D, const double *Vk, int k,
+                                   double beta, double beta_r, int first, double *Chat,
+                                   double *Rhat, double *C)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t n = 0; n < N; ++n) {
+        const double *f = F + (size_t)n * D;
+        double *c = C + (size_t)n * k;
+        double *rh = Rhat + (size_t)n * D;
+        double *ch = Chat + (size_t)n * k;
+        for (int j = 0; j < k; ++j) {
+            double s = 0.0;
+            for (int d = 0; d < D; ++d) s += f[d] * Vk[(size_t)d * k + j];
+            c[j] = s;
+        }
+        for (int d = 0; d < D; ++d) {
+            double s = 0.0;
+            for (int j = 0; j < k; ++j) s += c[j] * Vk[(size_t)d * k + j];
+            const double r = f[d] - s;
+            rh[d] = first ? r : beta_r * rh[d] + (1.0 - beta_r) * r;
+        }
+        for (int j = 0; j < k; ++j) ch[j] = first ? c[j] : beta * ch[j] + (1.0 - beta) * c[j];
+    }
+}
+
+/* ------------------------------------------------------------------------------------
+ * Other predictors on the principal coefficients (Sec. 5.3, Fig. 4(b)): the paper pairs its
+ * decomposition with predictors of the cited caching methods and does not restate them.  Two
+ * forecasts from the coefficients of the last order+1 full steps, hist[0] the newest,
+ * hist[i] the one i full steps earlier (each n values), for a cached step that lies
+ * u = (steps since the last full step) / (steps between full steps) intervals ahead:
+ *   backward differences   D^0 = hist[0],  D^i = D^{i-1}(newest) - D^{i-1}(one step earlier)
+ *   kind 1 ("taylor")  out = sum_i  u^i / i!  D^i
+ *        a Taylor expansion in the step offset whose derivatives are the backward differences
+ *        (the form of the cited cache-then-forecast method);
+ *   kind 2 ("newton")  out = sum_i  u (u+1) ... (u+i-1) / i!  D^i
+ *        Newton's backward-difference formula: the polynomial of degree `order` through the
+ *        last order+1 coefficients, evaluated u intervals past the newest.
+ * order = 0 is plain reuse of the newest coefficients (Eq. 3) for both kinds.
+ * ---------------------------------------------------------------------------------- */
+void oracle_forecast(const double *const *hist, int order, int64_t n, double u, int kind, double *out)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t e = 0; e < n; ++e) {
+        double d[8];                       /* d[j] = current difference anchored j steps back */
+        for (int j = 0; j <= order; ++j) d[j] = hist[j][e];
+        double acc = d[0], coef = 1.0;
+        for (int i = 1; i <= order; ++i) {
+            for (int j = 0; j + i <= order; ++j) d[j] = d[j] - d[j + 1];   /* now D^i at j steps back */
+            coef *= (kind == 1 ? u : (u + (double)(i - 1))) / (double)i;
+            acc += coef * d[0];
+        }
+        out[e] = acc;
+    }
+}
+
+/* ------------------------------------------------------------------------------------
+ * Left factors of Eq. 8:  U = F V_k diag(sigma_k)^{-1} = C diag(sigma_k)^{-1}, sigma_i the
+ * cached singular values (square roots of the Gram eigenvalues, Eq. 7).  A column whose
+ * sigma is zero carries no energy; it is set to zero instead of dividing.
+ * ---------------------------------------------------------------------------------- */
+void oracle_left_factors(const double *C, const double *sigma, int64_t N, int k, double *U)
+{
+    for (int64_t n = 0; n < N; ++n)
+        for (int j = 0; j < k; ++j)
+            U[(size_t)n * k + j] = sigma[j] > 0.0 ? C[(size_t)n * k + j] / sigma[j] : 0.0;
 }
 
 #ifdef _OPENMP

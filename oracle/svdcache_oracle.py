@@ -55,6 +55,12 @@ def _load():
             lib.oracle_full_step.restype = None
             lib.oracle_cached_step.argtypes = [_dp, _dp, _dp, i64, ci, ci, _dp]
             lib.oracle_cached_step.restype = None
+            lib.oracle_full_step_residual_ema.argtypes = [_dp, i64, ci, _dp, ci, cd, cd, ci, _dp, _dp, _dp]
+            lib.oracle_full_step_residual_ema.restype = None
+            lib.oracle_forecast.argtypes = [ctypes.POINTER(_dp), ci, i64, cd, ci, _dp]
+            lib.oracle_forecast.restype = None
+            lib.oracle_left_factors.argtypes = [_dp, _dp, i64, ci, _dp]
+            lib.oracle_left_factors.restype = None
             lib.oracle_threads.restype = ci
             lib.oracle_set_threads.argtypes = [ci]
             _lib = lib
@@ -160,3 +166,47 @@ def cached_step(Chat, Vk, R) -> np.ndarray:
     Fhat = np.empty((N, D))
     _load().oracle_cached_step(_p(Chat), _p(Vk), _p(R), N, D, k, _p(Fhat))
     return Fhat
+
+
+def full_step_residual_ema(F, Vk, beta: float, beta_r: float, Chat_prev=None, Rhat_prev=None):
+    """Full step whose stored residual is an EMA of the residuals (ablation, Fig. 4(c)).
+    Returns (C, Rhat, Chat); ``Chat_prev is None`` marks the first one."""
+    F = _f64(F)
+    Vk = _f64(Vk)
+    N, D = F.shape
+    k = Vk.shape[1]
+    first = Chat_prev is None
+    Chat = np.zeros((N, k)) if first else _f64(Chat_prev).copy()
+    Rhat = np.zeros((N, D)) if first else _f64(Rhat_prev).copy()
+    C = np.empty((N, k))
+    _load().oracle_full_step_residual_ema(_p(F), N, D, _p(Vk), k, float(beta), float(beta_r), int(first),
+                                          _p(Chat), _p(Rhat), _p(C))
+    return C, Rhat, Chat
+
+
+FORECAST_KINDS = {"taylor": 1, "newton": 2}
+
+
+def forecast(history, u: float, kind: str = "taylor") -> np.ndarray:
+    """Forecast of the coefficients ``u`` intervals past the newest full step from the list
+    ``history`` (newest first; its length - 1 is the order)."""
+    hist = [_f64(h) for h in history]
+    order = len(hist) - 1
+    if not 0 <= order <= 7:
+        raise ValueError("order must be in 0..7")
+    n = hist[0].size
+    assert all(h.shape == hist[0].shape for h in hist)
+    ptrs = (_dp * (order + 1))(*[_p(h) for h in hist])
+    out = np.empty_like(hist[0])
+    _load().oracle_forecast(ptrs, order, n, float(u), FORECAST_KINDS[kind], _p(out))
+    return out
+
+
+def left_factors(C, sigma) -> np.ndarray:
+    """U = C diag(sigma)^-1 (Eq. 8)."""
+    C = _f64(C)
+    sigma = _f64(sigma)
+    N, k = C.shape
+    U = np.empty((N, k))
+    _load().oracle_left_factors(_p(C), _p(sigma), N, k, _p(U))
+    return U
