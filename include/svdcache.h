@@ -61,6 +61,11 @@ extern "C" {
 #define SVDCACHE_F32   0
 #define SVDCACHE_BF16  1
 
+/* Predictors of the principal coefficients on cached steps (Sec. 3.4; Sec. 5.3, Fig. 4(b)). */
+#define SVDCACHE_PREDICT_EMA     0  /* the method's own: the EMA state of Eq. 11                          */
+#define SVDCACHE_PREDICT_TAYLOR  1  /* Taylor expansion in the step offset, backward-difference derivatives */
+#define SVDCACHE_PREDICT_NEWTON  2  /* polynomial through the last order+1 full steps (Newton backward form) */
+
 /* Text for a status code (static storage, never NULL). */
 SVDCACHE_API const char *svdcache_status_string(int status);
 
@@ -167,13 +172,11 @@ SVDCACHE_API int svdcache_basis_prepare(const float *Vk, int D, int k, int dtype
 
 /* ---------------------------------------------------------------------------------
  * Per-block cache state, a caller-owned flat device buffer (checkpoint = memcpy):
- *   header (256 B) | Chat fp32 [N x k] | Chat operand copy | step scratch | R dtype [N x D]   (dense, no pitch)
+ *   header (256 B) | Chat fp32 [N x k] | Chat operand copy | R dtype [N x D]   (dense, no pitch)
  * The operand copy exists only for dtype = SVDCACHE_BF16: Chat as two bf16 arrays [N x k],
  * hi = bf16(Chat) and lo = bf16(Chat - hi), which every full step rewrites together with
  * Chat and the cached step feeds to the tensor cores as they are (hi + lo carries ~16
- * mantissa bits).  The step scratch (bf16 mode only) belongs to the full step: this step's
- * coefficients C in the same split form, and four words per 128-row tile.  Offsets of Chat
- * and R come from svdcache_state_layout.
+ * mantissa bits).  Offsets of Chat and R come from svdcache_state_layout.
  * The header counts the full steps the state has seen and carries a sticky device
  * status word.  svdcache_state_reset must be called once before first use (and again to
  * start a new sampling run): it clears the counter, so the next full step initialises
@@ -204,8 +207,8 @@ SVDCACHE_API int svdcache_full_step(const void *F, int64_t ld, const void *basis
 /* ---------------------------------------------------------------------------------
  * Cached step (Sec. 3.5): Fhat = Chat V_k^T + R.  The EMA state changes only at full
  * steps, so every cached step until the next full step returns the same Fhat;
- * `steps_since_full` is accepted for predictors that extrapolate and is ignored by the
- * EMA.  If the state has seen no full step the kernel writes nothing and records
+ * `steps_since_full` is ignored by the EMA (the predictors that use it are the
+ * svdcache_cached_step_forecast calls below).  If the state has seen no full step the kernel writes nothing and records
  * SVDCACHE_ERR_STATE in the state header (read it with svdcache_state_query).
  *   Fhat   device, out, N x D, pitch ld
  * ------------------------------------------------------------------------------- */
@@ -227,6 +230,80 @@ SVDCACHE_API int svdcache_cached_step_batched(int nblocks, const void *state, si
                                  const void *basis, size_t basis_stride, void *Fhat,
                                  int64_t ld, size_t Fhat_stride, int64_t N, int D, int k,
                                  int dtype, int steps_since_full, void *stream);
+
+/* ---------------------------------------------------------------------------------
+ * Blocks of different rank in one call (Eq. 6: the rank follows each block's spectrum, see
+ * svdcache_rank_for_energy).  k_per_block is a HOST array of nblocks ranks; block b's basis and
+ * state buffers are laid out for k_per_block[b] and sit b * stride bytes from the first (the
+ * strides must cover the largest of them; C_out rows are k_per_block[b] wide).  Consecutive
+ * blocks of equal rank go out as one batched launch; everything else is as in the batched
+ * forms above.
+ * ------------------------------------------------------------------------------- */
+SVDCACHE_API int svdcache_full_step_ranked_batched(int nblocks, const void *F, int64_t ld, size_t F_stride,
+                                      const void *basis, size_t basis_stride, void *state,
+                                      size_t state_stride, float *C_out, size_t C_stride, int64_t N,
+                                      int D, const int *k_per_block, int dtype, float beta,
+                                      void *stream);
+SVDCACHE_API int svdcache_cached_step_ranked_batched(int nblocks, const void *state, size_t state_stride,
+                                        const void *basis, size_t basis_stride, void *Fhat,
+                                        int64_t ld, size_t Fhat_stride, int64_t N, int D,
+                                        const int *k_per_block, int dtype, int steps_since_full,
+                                        void *stream);
+
+/* ---------------------------------------------------------------------------------
+ * Other predictors on the principal coefficients (Sec. 5.3, Fig. 4(b)): the decomposition
+ * paired with a predictor that extrapolates inside the interval.  The caller keeps the
+ * coefficients C of the last order+1 full steps (the C_out of svdcache_full_step) and hands
+ * them over newest first; the residual is still the stored R (Sec. 3.5):
+ *     Fhat = (sum_j w_j C_{n-j}) V_k^T + R,      u = steps_since_full / interval,
+ *     backward differences D^i of the history, and
+ *     SVDCACHE_PREDICT_TAYLOR   sum_i u^i / i! D^i
+ *     SVDCACHE_PREDICT_NEWTON   sum_i u (u+1) ... (u+i-1) / i! D^i   (exact for polynomials of degree <= order)
+ *     SVDCACHE_PREDICT_EMA      ignores the history: the plain cached step.
+ * order 0 of either is plain reuse of the newest coefficients (Eq. 3).  order <= 7.
+ *   svdcache_forecast_weights  host: the order+1 weights w_j (newest first) into w
+ *   svdcache_forecast_bytes    host: size of the forecast buffer for N x k coefficients
+ *   C_hist     HOST array of order+1 DEVICE pointers, each N x k fp32 (block b at + b*C_stride bytes)
+ *   forecast   device scratch, 256-byte aligned, >= svdcache_forecast_bytes (block b at
+ *              + b*forecast_stride): receives the forecast (fp32, then its split-bf16 pair)
+ * Two launches: the forecast (N k work), then the cached-step kernel reading it.  The state is
+ * only read.  Errors as svdcache_cached_step.
+ * ------------------------------------------------------------------------------- */
+SVDCACHE_API int svdcache_forecast_weights(int predictor, int order, int steps_since_full, int interval,
+                              double *w /* host, out, order+1 */);
+SVDCACHE_API int svdcache_forecast_bytes(int64_t N, int k, size_t *bytes /* host, out */);
+SVDCACHE_API int svdcache_cached_step_forecast_batched(int nblocks, const void *state, size_t state_stride,
+                                          const void *basis, size_t basis_stride, void *Fhat,
+                                          int64_t ld, size_t Fhat_stride, int64_t N, int D, int k,
+                                          int dtype, const float *const *C_hist, size_t C_stride,
+                                          int predictor, int order, int steps_since_full,
+                                          int interval, void *forecast, size_t forecast_stride,
+                                          void *stream);
+
+/* ---------------------------------------------------------------------------------
+ * Ablation of Sec. 4.5 (Fig. 4(c)): the stored residual as an EMA of the residuals,
+ *     R <- F - C V_k^T on the first full step, else beta_r R + (1 - beta_r)(F - C V_k^T).
+ * beta_r = 0 is svdcache_full_step itself (the method: the residual is reused as it is);
+ * beta = beta_r = 0 is "reuse on both" (Eq. 3); beta, beta_r > 0 is "EMA on both".  With
+ * beta_r > 0 the step reads the old R as well (N D more elements than the method's step) and
+ * runs on the CUDA-core kernels.  Arguments as svdcache_full_step_batched.
+ * ------------------------------------------------------------------------------- */
+SVDCACHE_API int svdcache_full_step_residual_ema_batched(int nblocks, const void *F, int64_t ld,
+                                            size_t F_stride, const void *basis, size_t basis_stride,
+                                            void *state, size_t state_stride, float *C_out,
+                                            size_t C_stride, int64_t N, int D, int k, int dtype,
+                                            float beta, float beta_r, void *stream);
+
+/* ---------------------------------------------------------------------------------
+ * The cached singular values and the left factors of Eq. 7 - Eq. 8.
+ *   svdcache_singular_values  sigma_i = sqrt(lambda_i) of the calibration spectrum (device arrays of k)
+ *   svdcache_left_factors     U = C diag(sigma)^-1 (Eq. 8), C and U device N x k fp32; a column whose
+ *                             sigma is 0 is set to 0.  (The step kernels never form U: sigma cancels
+ *                             between Eq. 8 and Eq. 9.)
+ * ------------------------------------------------------------------------------- */
+SVDCACHE_API int svdcache_singular_values(const double *lambda, int k, double *sigma, void *stream);
+SVDCACHE_API int svdcache_left_factors(const float *C, const double *sigma, int64_t N, int k, float *U,
+                          void *stream);
 
 /* ---------------------------------------------------------------------------------
  * Introspection for benchmarks and tests (host only).

@@ -51,6 +51,18 @@ SIGNATURES = {
     "svdcache_set_path": (_ci, [_ci]),
     "svdcache_last_path": (_ci, []),
     "svdcache_selftest_wait_timeout": (_ci, [_vp, _i64, _vp]),
+    "svdcache_full_step_ranked_batched": (_ci, [_ci, _vp, _i64, _sz, _vp, _sz, _vp, _sz, _vp, _sz, _i64, _ci,
+                                                ctypes.POINTER(_ci), _ci, ctypes.c_float, _vp]),
+    "svdcache_cached_step_ranked_batched": (_ci, [_ci, _vp, _sz, _vp, _sz, _vp, _i64, _sz, _i64, _ci,
+                                                  ctypes.POINTER(_ci), _ci, _ci, _vp]),
+    "svdcache_forecast_weights": (_ci, [_ci, _ci, _ci, _ci, ctypes.POINTER(ctypes.c_double)]),
+    "svdcache_forecast_bytes": (_ci, [_i64, _ci, _szp]),
+    "svdcache_cached_step_forecast_batched": (_ci, [_ci, _vp, _sz, _vp, _sz, _vp, _i64, _sz, _i64, _ci, _ci, _ci,
+                                                    ctypes.POINTER(_vp), _sz, _ci, _ci, _ci, _ci, _vp, _sz, _vp]),
+    "svdcache_full_step_residual_ema_batched": (_ci, [_ci, _vp, _i64, _sz, _vp, _sz, _vp, _sz, _vp, _sz, _i64, _ci,
+                                                      _ci, _ci, ctypes.c_float, ctypes.c_float, _vp]),
+    "svdcache_singular_values": (_ci, [_vp, _ci, _vp, _vp]),
+    "svdcache_left_factors": (_ci, [_vp, _vp, _i64, _ci, _vp, _vp]),
 }
 
 
@@ -294,6 +306,94 @@ def svdcache_last_path() -> int:
 
 def svdcache_selftest_wait_timeout(state: torch.Tensor, limit_cycles: int, stream=None) -> None:
     _check(lib().svdcache_selftest_wait_timeout(_ptr(state), int(limit_cycles), _stream(stream)), "selftest_wait_timeout")
+
+
+PREDICT_EMA, PREDICT_TAYLOR, PREDICT_NEWTON = 0, 1, 2
+
+
+def svdcache_forecast_weights(predictor: int, order: int, steps_since_full: int, interval: int):
+    w = (ctypes.c_double * (order + 1))()
+    _check(lib().svdcache_forecast_weights(predictor, order, steps_since_full, interval, w), "forecast_weights")
+    return list(w)
+
+
+def svdcache_forecast_bytes(N: int, k: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().svdcache_forecast_bytes(N, k, ctypes.byref(out)), "forecast_bytes")
+    return int(out.value)
+
+
+def svdcache_cached_step_forecast_batched(state: torch.Tensor, basis: torch.Tensor, Fhat: torch.Tensor, k: int, history,
+                                  predictor: int, steps_since_full: int, interval: int, forecast=None, stream=None):
+    """Cached step with the coefficients forecast from `history` (list of N x k fp32 device tensors --
+    or [blocks, N, k] for a batched Fhat [blocks, N, D] -- newest first; its length - 1 is the order).
+    Returns the forecast buffer (allocated here unless given)."""
+    batched = Fhat.dim() == 3
+    nb = Fhat.shape[0] if batched else 1
+    N, D = Fhat.shape[-2:]
+    assert Fhat.stride(-1) == 1
+    order = len(history) - 1
+    fbytes = svdcache_forecast_bytes(N, k)
+    if forecast is None:
+        forecast = torch.empty(nb, fbytes, dtype=torch.uint8, device=Fhat.device) if batched else _bytes_buffer(fbytes, Fhat.device)
+    ptrs = (_vp * (order + 1))(*[_ptr(h) for h in history])
+    eb = Fhat.element_size()
+    _check(lib().svdcache_cached_step_forecast_batched(
+        nb, _ptr(state), state.stride(0) if batched else 0, _ptr(basis), basis.stride(0) if batched else 0, _ptr(Fhat),
+        Fhat.stride(-2), Fhat.stride(0) * eb if batched else 0, N, D, k, _dt(Fhat), ptrs,
+        history[0].stride(0) * 4 if batched else 0, predictor, order, int(steps_since_full), int(interval), _ptr(forecast),
+        forecast.stride(0) if batched else 0, _stream(stream)), "cached_step_forecast")
+    return forecast
+
+
+def svdcache_full_step_residual_ema_batched(F: torch.Tensor, basis: torch.Tensor, state: torch.Tensor, k: int, beta: float,
+                                    beta_r: float, C_out: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Full step whose stored residual is an EMA of the residuals (ablation); F is [N, D] or [blocks, N, D]."""
+    batched = F.dim() == 3
+    nb = F.shape[0] if batched else 1
+    N, D = F.shape[-2:]
+    eb = F.element_size()
+    _check(lib().svdcache_full_step_residual_ema_batched(
+        nb, _ptr(F), F.stride(-2), F.stride(0) * eb if batched else 0, _ptr(basis), basis.stride(0) if batched else 0,
+        _ptr(state), state.stride(0) if batched else 0, _ptr(C_out) if C_out is not None else None,
+        C_out.stride(0) * 4 if (batched and C_out is not None) else 0, N, D, k, _dt(F), float(beta), float(beta_r),
+        _stream(stream)), "full_step_residual_ema")
+
+
+def svdcache_full_step_ranked_batched(F: torch.Tensor, bases: torch.Tensor, states: torch.Tensor, ranks, beta: float,
+                              C_out: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Batched full step over blocks of different rank: F [blocks, N, D], bases / states [blocks, bytes]
+    (each block's buffer laid out for its own rank), C_out [blocks, N, kmax] (row b*... holds N x k_b dense)."""
+    nb, N, D = F.shape
+    arr = (_ci * nb)(*[int(r) for r in ranks])
+    _check(lib().svdcache_full_step_ranked_batched(
+        nb, _ptr(F), F.stride(1), F.stride(0) * F.element_size(), _ptr(bases), bases.stride(0), _ptr(states),
+        states.stride(0), _ptr(C_out) if C_out is not None else None, C_out.stride(0) * 4 if C_out is not None else 0,
+        N, D, arr, _dt(F), float(beta), _stream(stream)), "full_step_ranked")
+
+
+def svdcache_cached_step_ranked_batched(states: torch.Tensor, bases: torch.Tensor, Fhat: torch.Tensor, ranks,
+                                steps_since_full: int = 1, stream=None) -> None:
+    nb, N, D = Fhat.shape
+    arr = (_ci * nb)(*[int(r) for r in ranks])
+    _check(lib().svdcache_cached_step_ranked_batched(
+        nb, _ptr(states), states.stride(0), _ptr(bases), bases.stride(0), _ptr(Fhat), Fhat.stride(1),
+        Fhat.stride(0) * Fhat.element_size(), N, D, arr, _dt(Fhat), int(steps_since_full), _stream(stream)),
+        "cached_step_ranked")
+
+
+def svdcache_singular_values(lam: torch.Tensor, stream=None) -> torch.Tensor:
+    sigma = torch.empty_like(lam)
+    _check(lib().svdcache_singular_values(_ptr(lam), lam.numel(), _ptr(sigma), _stream(stream)), "singular_values")
+    return sigma
+
+
+def svdcache_left_factors(C: torch.Tensor, sigma: torch.Tensor, stream=None) -> torch.Tensor:
+    N, k = C.shape
+    assert C.is_contiguous() and C.dtype == torch.float32 and sigma.dtype == torch.float64
+    U = torch.empty_like(C)
+    _check(lib().svdcache_left_factors(_ptr(C), _ptr(sigma), N, k, _ptr(U), _stream(stream)), "left_factors")
+    return U
 
 
 # ---------------------------------------------------------- views for tests/tools ---

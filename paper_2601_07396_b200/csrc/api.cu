@@ -42,6 +42,12 @@ static int dispatch(const StepArgs &a_in, bool full, cudaStream_t s) {
     const int want = g_path.load();
     const bool can_umma = umma_supported(a, full);
     if (want == 2 && !can_umma) return SVDCACHE_ERR_BAD_SHAPE;
+    // the residual EMA of the ablation is a read-modify-write of R: it runs on the CUDA-core kernels
+    if (full && a.beta_r > 0.0f) {
+        if (want == 2) return SVDCACHE_ERR_BAD_SHAPE;
+        g_last_path.store(1);
+        return simt_full_step(a, s);
+    }
     const bool use_umma = (want == 2) || (want == 0 && can_umma);
     g_last_path.store(use_umma ? 2 : 1);
     if (use_umma) return full ? umma_full_step(a, s) : umma_cached_step(a, s);
@@ -296,6 +302,113 @@ int svdcache_cached_step_batched(int nblocks, const void *state, size_t state_st
     int rc = check_step(a, false);
     if (rc) return rc;
     return dispatch(a, false, (cudaStream_t)stream);
+}
+
+int svdcache_full_step_residual_ema_batched(int nblocks, const void *F, int64_t ld, size_t F_stride,
+                                            const void *basis, size_t basis_stride, void *state,
+                                            size_t state_stride, float *C_out, size_t C_stride, int64_t N,
+                                            int D, int k, int dtype, float beta, float beta_r, void *stream) {
+    if (!(beta_r >= 0.0f && beta_r <= 1.0f)) return SVDCACHE_ERR_INVALID_ARG;
+    StepArgs a{};
+    a.F = F; a.ld = ld; a.F_stride = F_stride; a.basis = basis; a.basis_stride = basis_stride;
+    a.state = state; a.state_stride = state_stride; a.C_out = C_out; a.C_stride = C_stride;
+    a.N = N; a.D = D; a.k = k; a.dtype = dtype; a.beta = beta; a.beta_r = beta_r; a.nblocks = nblocks;
+    int rc = check_step(a, true);
+    if (rc) return rc;
+    return dispatch(a, true, (cudaStream_t)stream);
+}
+
+int svdcache_forecast_weights(int predictor, int order, int steps_since_full, int interval, double *w) {
+    if (!w || interval < 1 || steps_since_full < 0) return SVDCACHE_ERR_INVALID_ARG;
+    return forecast_weights(predictor, order, (double)steps_since_full / (double)interval, w);
+}
+
+int svdcache_forecast_bytes(int64_t N, int k, size_t *bytes) {
+    if (!bytes) return SVDCACHE_ERR_INVALID_ARG;
+    if (N < 1 || k < 8 || k > 256 || (k % 8) != 0) return SVDCACHE_ERR_BAD_SHAPE;
+    *bytes = forecast_layout(N, k).total;
+    return SVDCACHE_OK;
+}
+
+int svdcache_cached_step_forecast_batched(int nblocks, const void *state, size_t state_stride, const void *basis,
+                                          size_t basis_stride, void *Fhat, int64_t ld, size_t Fhat_stride,
+                                          int64_t N, int D, int k, int dtype, const float *const *C_hist,
+                                          size_t C_stride, int predictor, int order, int steps_since_full,
+                                          int interval, void *forecast, size_t forecast_stride, void *stream) {
+    StepArgs a{};
+    a.Fhat = Fhat; a.ld = ld; a.Fhat_stride = Fhat_stride; a.basis = basis; a.basis_stride = basis_stride;
+    a.state = const_cast<void *>(state); a.state_stride = state_stride;
+    a.N = N; a.D = D; a.k = k; a.dtype = dtype; a.nblocks = nblocks;
+    int rc = check_step(a, false);
+    if (rc) return rc;
+    if (predictor == SVDCACHE_PREDICT_EMA) return dispatch(a, false, (cudaStream_t)stream);   // the state's own forecast
+    if (!C_hist || !forecast || interval < 1 || steps_since_full < 0) return SVDCACHE_ERR_INVALID_ARG;
+    double w[8];
+    rc = forecast_weights(predictor, order, (double)steps_since_full / (double)interval, w);
+    if (rc) return rc;
+    for (int j = 0; j <= order; ++j) {
+        if (!C_hist[j]) return SVDCACHE_ERR_INVALID_ARG;
+        if (!aligned16(C_hist[j])) return SVDCACHE_ERR_BAD_ALIGN;
+    }
+    if ((reinterpret_cast<uintptr_t>(forecast) & 255u) != 0) return SVDCACHE_ERR_BAD_ALIGN;
+    if (nblocks > 1) {
+        if (C_stride % 256 != 0 || forecast_stride % 256 != 0) return SVDCACHE_ERR_BAD_ALIGN;
+        if (C_stride < (size_t)N * k * 4 || forecast_stride < forecast_layout(N, k).total) return SVDCACHE_ERR_BAD_SHAPE;
+    }
+    rc = forecast_launch(C_hist, C_stride, w, order, N, k, dtype, nblocks, forecast, forecast_stride, (cudaStream_t)stream);
+    if (rc) return rc;
+    a.coef = forecast;
+    a.coef_stride = forecast_stride;
+    return dispatch(a, false, (cudaStream_t)stream);
+}
+
+int svdcache_singular_values(const double *lambda, int k, double *sigma, void *stream) {
+    if (!lambda || !sigma) return SVDCACHE_ERR_INVALID_ARG;
+    if (k < 1 || k > 16384) return SVDCACHE_ERR_BAD_SHAPE;
+    return sigma_launch(lambda, k, sigma, (cudaStream_t)stream);
+}
+
+int svdcache_left_factors(const float *C, const double *sigma, int64_t N, int k, float *U, void *stream) {
+    if (!C || !sigma || !U) return SVDCACHE_ERR_INVALID_ARG;
+    if (N < 1 || k < 1 || k > 16384) return SVDCACHE_ERR_BAD_SHAPE;
+    return left_factors_launch(C, sigma, N, k, U, (cudaStream_t)stream);
+}
+
+/* Blocks of different rank in one call: consecutive blocks of equal rank form one batched launch. */
+int svdcache_full_step_ranked_batched(int nblocks, const void *F, int64_t ld, size_t F_stride, const void *basis,
+                                      size_t basis_stride, void *state, size_t state_stride, float *C_out,
+                                      size_t C_stride, int64_t N, int D, const int *k_per_block, int dtype,
+                                      float beta, void *stream) {
+    if (!k_per_block || nblocks < 1) return SVDCACHE_ERR_INVALID_ARG;
+    for (int b0 = 0; b0 < nblocks;) {
+        int b1 = b0 + 1;
+        while (b1 < nblocks && k_per_block[b1] == k_per_block[b0]) ++b1;
+        const int rc = svdcache_full_step_batched(
+            b1 - b0, (const char *)F + (size_t)b0 * F_stride, ld, F_stride, (const char *)basis + (size_t)b0 * basis_stride,
+            basis_stride, (char *)state + (size_t)b0 * state_stride, state_stride,
+            C_out ? reinterpret_cast<float *>((char *)C_out + (size_t)b0 * C_stride) : nullptr, C_stride, N, D,
+            k_per_block[b0], dtype, beta, stream);
+        if (rc) return rc;
+        b0 = b1;
+    }
+    return SVDCACHE_OK;
+}
+
+int svdcache_cached_step_ranked_batched(int nblocks, const void *state, size_t state_stride, const void *basis,
+                                        size_t basis_stride, void *Fhat, int64_t ld, size_t Fhat_stride, int64_t N,
+                                        int D, const int *k_per_block, int dtype, int steps_since_full, void *stream) {
+    if (!k_per_block || nblocks < 1) return SVDCACHE_ERR_INVALID_ARG;
+    for (int b0 = 0; b0 < nblocks;) {
+        int b1 = b0 + 1;
+        while (b1 < nblocks && k_per_block[b1] == k_per_block[b0]) ++b1;
+        const int rc = svdcache_cached_step_batched(
+            b1 - b0, (const char *)state + (size_t)b0 * state_stride, state_stride,
+            (const char *)basis + (size_t)b0 * basis_stride, basis_stride, (char *)Fhat + (size_t)b0 * Fhat_stride, ld,
+            Fhat_stride, N, D, k_per_block[b0], dtype, steps_since_full, stream);
+        if (rc) return rc;
+        b0 = b1;
+    }
+    return SVDCACHE_OK;
 }
 
 int svdcache_full_step(const void *F, int64_t ld, const void *basis, void *state, float *C_out, int64_t N,

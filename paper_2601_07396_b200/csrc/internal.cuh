@@ -88,6 +88,9 @@ struct StepArgs {
     int64_t N;
     int D, k, dtype, nblocks;
     float beta;
+    float beta_r;           // full step: EMA weight of the stored residual (0 = the residual is replaced, Sec. 3.5)
+    const void *coef;       // cached step: forecast buffer (fp32 | hi | lo, forecast_layout) to take the
+    size_t coef_stride;     //   coefficients from instead of the state's Chat; null = the state's own
 };
 
 // launch bookkeeping (api.cu)
@@ -104,6 +107,17 @@ bool umma_supported(const StepArgs &a, bool full);
 int umma_full_step(const StepArgs &a, cudaStream_t s);
 int umma_cached_step(const StepArgs &a, cudaStream_t s);
 int umma_wait_selftest(void *state, long long limit_cycles, cudaStream_t s);
+
+// forecasts and coefficient-side helpers (forecast.cu)
+struct ForecastLayout {
+    size_t f32, hi, lo, total;
+};
+ForecastLayout forecast_layout(int64_t N, int k);
+int forecast_weights(int predictor, int order, double u, double *w);
+int forecast_launch(const float *const *hist, size_t hist_stride, const double *w, int order, int64_t N, int k,
+                    int dtype, int nblocks, void *out, size_t out_stride, cudaStream_t s);
+int sigma_launch(const double *lambda, int k, double *sigma, cudaStream_t s);
+int left_factors_launch(const float *C, const double *sigma, int64_t N, int k, float *U, cudaStream_t s);
 
 // basis (basis.cu)
 int basis_prepare(const float *Vk, int D, int k, int dtype, void *basis, cudaStream_t s);

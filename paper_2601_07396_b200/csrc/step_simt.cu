@@ -91,7 +91,12 @@ simt_full_kernel(StepArgs a, size_t v_off, size_t vt_off, StateLayout SL) {
 #pragma unroll
         for (int r = 0; r < kRows; ++r) {
             const int64_t n = row0 + r;
-            if (n < a.N) R[n * D + d] = from_acc<T, Acc>((Acc)Fs[(size_t)r * D + d] - acc[r]);
+            if (n < a.N) {
+                Acc res = (Acc)Fs[(size_t)r * D + d] - acc[r];
+                // ablation (Sec. 4.5): the stored residual as an EMA of the residuals
+                if (a.beta_r > 0.0f && !first) res = (Acc)a.beta_r * (Acc)ld_as_float(R + n * D + d) + (Acc)(1.0f - a.beta_r) * res;
+                R[n * D + d] = from_acc<T, Acc>(res);
+            }
         }
     }
 
@@ -121,7 +126,9 @@ simt_cached_kernel(StepArgs a, size_t vt_off, size_t chat_off, size_t r_off) {
     char *state = (char *)a.state + (size_t)b * a.state_stride;
     const BT *Vt = reinterpret_cast<const BT *>(basis + vt_off);
     StateHeader *hdr = reinterpret_cast<StateHeader *>(state);
-    const float *Chat = reinterpret_cast<const float *>(state + chat_off);
+    // the coefficients come from the state's EMA, or from a forecast buffer (its fp32 part first)
+    const float *Chat = a.coef ? reinterpret_cast<const float *>((const char *)a.coef + (size_t)b * a.coef_stride)
+                               : reinterpret_cast<const float *>(state + chat_off);
     const T *R = reinterpret_cast<const T *>(state + r_off);
     T *Fhat = reinterpret_cast<T *>((char *)a.Fhat + (size_t)b * a.Fhat_stride);
 

@@ -1283,11 +1283,14 @@ int umma_cached_step(const StepArgs &a, cudaStream_t s) {
     rc = make_map(&tm_v, (const char *)a.basis + BL.v_bf16, a.k, a.D, a.nblocks, (uint64_t)a.k * 2, a.basis_stride,
                   p.kb_elems, p.gc * kTileCols);
     if (rc) return rc;
-    rc = make_map(&tm_ahi, (const char *)a.state + SL.op_hi, a.k, a.N, a.nblocks, (uint64_t)a.k * 2, a.state_stride,
-                  p.kb_elems, kTileRows);
+    // the operand: the split pair of the state's Chat, or that of a forecast buffer
+    const ForecastLayout FL = forecast_layout(a.N, a.k);
+    const char *op_hi = a.coef ? (const char *)a.coef + FL.hi : (const char *)a.state + SL.op_hi;
+    const char *op_lo = a.coef ? (const char *)a.coef + FL.lo : (const char *)a.state + SL.op_lo;
+    const size_t op_stride = a.coef ? a.coef_stride : a.state_stride;
+    rc = make_map(&tm_ahi, op_hi, a.k, a.N, a.nblocks, (uint64_t)a.k * 2, op_stride, p.kb_elems, kTileRows);
     if (rc) return rc;
-    rc = make_map(&tm_alo, (const char *)a.state + SL.op_lo, a.k, a.N, a.nblocks, (uint64_t)a.k * 2, a.state_stride,
-                  p.kb_elems, kTileRows);
+    rc = make_map(&tm_alo, op_lo, a.k, a.N, a.nblocks, (uint64_t)a.k * 2, op_stride, p.kb_elems, kTileRows);
     if (rc) return rc;
     rc = make_map(&tm_out, a.Fhat, a.D, a.N, a.nblocks, (uint64_t)a.ld * 2, a.Fhat_stride, kTileCols, kSlabRows);
     if (rc) return rc;

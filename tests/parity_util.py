@@ -42,10 +42,11 @@ def check_close(name, got, ref, dtype, rms_f, coeff=0):
         # (2^-9 |x|) however it was computed, which passes 2e-2 * rms(F) once |x| > 10 rms(F);
         # among the 1e8 elements sampled at the full FLUX size a few are that large.
         err = np.abs(got - ref)
-        bound_el = np.maximum(tol["maxabs"] * rms_f, 2.0 ** -8 * np.abs(ref))
+        ulp = np.exp2(np.floor(np.log2(np.maximum(np.abs(ref), 1e-30))) - 7.0)   # bf16: 8 significant bits
+        bound_el = np.maximum(tol["maxabs"] * rms_f, ulp)
         worst = int(np.argmax(err - bound_el))
         assert (err <= bound_el).all(), (f"{name}: element error {err.flat[worst]:.3e} > "
-                                        f"max({tol['maxabs']}*rms(F)={tol['maxabs'] * rms_f:.3e}, 2^-8*|ref|={2.0 ** -8 * abs(ref.flat[worst]):.3e})")
+                                        f"max({tol['maxabs']}*rms(F)={tol['maxabs'] * rms_f:.3e}, ulp(ref)={ulp.flat[worst]:.3e})")
     return rel
 
 
