@@ -117,6 +117,22 @@ SVDCACHE_API int svdcache_calibrate(const void *Fstack, int64_t M, int D, int64_
                        float *Vk, double *lambda, double *trace, double *info,
                        void *workspace, size_t workspace_bytes, void *stream);
 
+/* Where the Gram matrix sits in a calibration workspace (Eq. 4): D x D doubles, row-major, `offset`
+ * bytes from the start, complete between the last accumulate and the finish.  Row-sharded
+ * calibration over several GPUs: every rank begins and accumulates its own rows, the ranks sum
+ * this region (one all-reduce of D x D doubles), every rank finishes on the sum. */
+SVDCACHE_API int svdcache_calibrate_gram_region(int D, size_t *offset, size_t *bytes /* host, out */);
+
+/* Stability of the decomposition across "prompts" (Fig. 1(b)): similarity = cosine similarity x
+ * magnitude similarity (min / max of the two norms).  For the singular values sigma = sqrt(lambda)
+ * of two calibrations A and B: out[0] = cos(sigma_A, sigma_B) * min(|sigma_A|, |sigma_B|) / max(..).
+ * For the right singular vectors (unit columns, sign-free): column_cos[j] = |<v_j^A, v_j^B>|,
+ * out[1] = their mean.  VkA, VkB device D x k fp32, lambda device k doubles, column_cos device k
+ * doubles (out), out host 2 doubles.  Synchronises `stream`. */
+SVDCACHE_API int svdcache_basis_similarity(const float *VkA, const double *lambdaA, const float *VkB,
+                              const double *lambdaB, int D, int k, double *column_cos,
+                              double *out, void *stream);
+
 /* ---------------------------------------------------------------------------------
  * Calibration for callers that cannot allocate device memory.  (The paper has no
  * counterpart: this entry point exists for how the library gets embedded, not for the

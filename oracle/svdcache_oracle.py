@@ -210,3 +210,22 @@ def left_factors(C, sigma) -> np.ndarray:
     U = np.empty((N, k))
     _load().oracle_left_factors(_p(C), _p(sigma), N, k, _p(U))
     return U
+
+
+def basis_similarity(VA, lamA, VB, lamB):
+    """Stability of a decomposition across two calibrations (Fig. 1(b)): similarity = cosine
+    similarity x magnitude similarity (smaller norm / larger norm).  Returns (that of the singular
+    values sigma = sqrt(lambda), the mean over the columns of that of the right singular vectors,
+    the per-column values).  Singular vectors are sign-free, so their cosine enters in magnitude."""
+    VA, VB = _f64(VA), _f64(VB)
+    sa, sb = np.sqrt(np.maximum(_f64(lamA), 0.0)), np.sqrt(np.maximum(_f64(lamB), 0.0))
+
+    def sim(a, b, signed=True):
+        na, nb = np.linalg.norm(a), np.linalg.norm(b)
+        if na == 0.0 or nb == 0.0:
+            return 0.0
+        c = float(a @ b) / (na * nb)
+        return (c if signed else abs(c)) * min(na, nb) / max(na, nb)
+
+    cols = np.array([sim(VA[:, j], VB[:, j], signed=False) for j in range(VA.shape[1])])
+    return sim(sa, sb), float(cols.mean()), cols

@@ -61,6 +61,8 @@ SIGNATURES = {
                                                     ctypes.POINTER(_vp), _sz, _ci, _ci, _ci, _ci, _vp, _sz, _vp]),
     "svdcache_full_step_residual_ema_batched": (_ci, [_ci, _vp, _i64, _sz, _vp, _sz, _vp, _sz, _vp, _sz, _i64, _ci,
                                                       _ci, _ci, ctypes.c_float, ctypes.c_float, _vp]),
+    "svdcache_calibrate_gram_region": (_ci, [_ci, _szp, _szp]),
+    "svdcache_basis_similarity": (_ci, [_vp, _vp, _vp, _vp, _ci, _ci, _vp, ctypes.POINTER(ctypes.c_double), _vp]),
     "svdcache_singular_values": (_ci, [_vp, _ci, _vp, _vp]),
     "svdcache_left_factors": (_ci, [_vp, _vp, _i64, _ci, _vp, _vp]),
 }
@@ -380,6 +382,23 @@ def svdcache_cached_step_ranked_batched(states: torch.Tensor, bases: torch.Tenso
         nb, _ptr(states), states.stride(0), _ptr(bases), bases.stride(0), _ptr(Fhat), Fhat.stride(1),
         Fhat.stride(0) * Fhat.element_size(), N, D, arr, _dt(Fhat), int(steps_since_full), _stream(stream)),
         "cached_step_ranked")
+
+
+def svdcache_calibrate_gram_region(D: int):
+    off, nbytes = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    _check(lib().svdcache_calibrate_gram_region(D, ctypes.byref(off), ctypes.byref(nbytes)), "calibrate_gram_region")
+    return int(off.value), int(nbytes.value)
+
+
+def svdcache_basis_similarity(VkA: torch.Tensor, lamA: torch.Tensor, VkB: torch.Tensor, lamB: torch.Tensor, stream=None):
+    """(similarity of the singular values, mean similarity of the right singular vectors, per-column |cos|)."""
+    D, k = VkA.shape
+    assert VkB.shape == (D, k) and VkA.is_contiguous() and VkB.is_contiguous()
+    cols = torch.empty(k, dtype=torch.float64, device=VkA.device)
+    out = (ctypes.c_double * 2)()
+    _check(lib().svdcache_basis_similarity(_ptr(VkA), _ptr(lamA), _ptr(VkB), _ptr(lamB), D, k, _ptr(cols), out,
+                                           _stream(stream)), "basis_similarity")
+    return float(out[0]), float(out[1]), cols
 
 
 def svdcache_singular_values(lam: torch.Tensor, stream=None) -> torch.Tensor:

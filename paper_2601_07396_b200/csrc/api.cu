@@ -1,7 +1,9 @@
 // The extern "C" surface: argument validation, layout queries, dispatch to the kernels.
 #include <atomic>
 #include <cstdio>
+#include <cmath>
 #include <cstring>
+#include <vector>
 
 #include "internal.cuh"
 
@@ -165,6 +167,39 @@ int svdcache_calibrate(const void *Fstack, int64_t M, int D, int64_t ld, int dty
     rc = svdcache_calibrate_accumulate(Fstack, M, D, ld, dtype, ws, bytes, stream);
     if (rc) return rc;
     return svdcache_calibrate_finish(D, k, Vk, lambda, trace, info, ws, bytes, stream);
+}
+
+int svdcache_calibrate_gram_region(int D, size_t *offset, size_t *bytes) {
+    if (!offset || !bytes) return SVDCACHE_ERR_INVALID_ARG;
+    if (D < 8 || D > 16384 || (D % 8) != 0) return SVDCACHE_ERR_BAD_SHAPE;
+    *offset = calib_gram_offset();
+    *bytes = (size_t)D * D * sizeof(double);
+    return SVDCACHE_OK;
+}
+
+int svdcache_basis_similarity(const float *VkA, const double *lambdaA, const float *VkB, const double *lambdaB, int D,
+                              int k, double *column_cos, double *out, void *stream) {
+    if (!VkA || !VkB || !lambdaA || !lambdaB || !column_cos || !out) return SVDCACHE_ERR_INVALID_ARG;
+    if (D < 1 || k < 1 || k > D || k > 16384) return SVDCACHE_ERR_BAD_SHAPE;
+    int rc = column_cosines_launch(VkA, VkB, D, k, column_cos, (cudaStream_t)stream);
+    if (rc) return rc;
+    // the spectra are k numbers each: their statistic is formed on the host
+    std::vector<double> la(k), lb(k), cs(k);
+    rc = record_cuda(cudaMemcpyAsync(la.data(), lambdaA, k * sizeof(double), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    if (!rc) rc = record_cuda(cudaMemcpyAsync(lb.data(), lambdaB, k * sizeof(double), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    if (!rc) rc = record_cuda(cudaMemcpyAsync(cs.data(), column_cos, k * sizeof(double), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    if (!rc) rc = record_cuda(cudaStreamSynchronize((cudaStream_t)stream));
+    if (rc) return rc;
+    double ab = 0.0, aa = 0.0, bb = 0.0, mean = 0.0;
+    for (int i = 0; i < k; ++i) {
+        const double sa = la[i] > 0.0 ? std::sqrt(la[i]) : 0.0, sb = lb[i] > 0.0 ? std::sqrt(lb[i]) : 0.0;
+        ab += sa * sb; aa += sa * sa; bb += sb * sb;
+        mean += cs[i];
+    }
+    const double na = std::sqrt(aa), nb = std::sqrt(bb);
+    out[0] = (na > 0.0 && nb > 0.0) ? (ab / (na * nb)) * (na < nb ? na / nb : nb / na) : 0.0;
+    out[1] = mean / k;
+    return SVDCACHE_OK;
 }
 
 int svdcache_rank_for_energy(const double *lambda, int n, double trace, double tau, int *k_out) {

@@ -517,6 +517,8 @@ int calib_begin(int D, int k, void *ws, cudaStream_t s) {
     return check_last_launch();
 }
 
+size_t calib_gram_offset() { return kHeaderBytes; }
+
 int calib_accumulate(const void *F, int64_t M, int D, int64_t ld, int dtype, void *ws, cudaStream_t s) {
     // G sits at a fixed offset whatever k is
     char *w = (char *)ws;

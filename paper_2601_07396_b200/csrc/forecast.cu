@@ -58,7 +58,36 @@ __global__ void __launch_bounds__(256) left_factors_kernel(const float *C, const
     }
 }
 
+// |<a_j, b_j>| of the unit columns j of two D x k bases (one CTA per column, fixed reduction order)
+__global__ void __launch_bounds__(256) column_cosines_kernel(const float *A, const float *B, int D, int k, double *out) {
+    __shared__ double part[256];
+    const int j = blockIdx.x;
+    double ab = 0.0, aa = 0.0, bb = 0.0;
+    for (int d = threadIdx.x; d < D; d += 256) {
+        const double a = (double)A[(size_t)d * k + j], b = (double)B[(size_t)d * k + j];
+        ab += a * b; aa += a * a; bb += b * b;
+    }
+    double r[3] = {ab, aa, bb};
+    for (int q = 0; q < 3; ++q) {
+        part[threadIdx.x] = r[q];
+        __syncthreads();
+        for (int sft = 128; sft > 0; sft >>= 1) {
+            if ((int)threadIdx.x < sft) part[threadIdx.x] += part[threadIdx.x + sft];
+            __syncthreads();
+        }
+        r[q] = part[0];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) out[j] = (r[1] > 0.0 && r[2] > 0.0) ? fabs(r[0]) / sqrt(r[1] * r[2]) : 0.0;
+}
+
 }  // namespace
+
+int column_cosines_launch(const float *A, const float *B, int D, int k, double *out, cudaStream_t s) {
+    column_cosines_kernel<<<k, 256, 0, s>>>(A, B, D, k, out);
+    count_launch();
+    return check_last_launch();
+}
 
 ForecastLayout forecast_layout(int64_t N, int k) {
     ForecastLayout L;

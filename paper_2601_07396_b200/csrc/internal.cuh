@@ -118,12 +118,14 @@ int forecast_launch(const float *const *hist, size_t hist_stride, const double *
                     int dtype, int nblocks, void *out, size_t out_stride, cudaStream_t s);
 int sigma_launch(const double *lambda, int k, double *sigma, cudaStream_t s);
 int left_factors_launch(const float *C, const double *sigma, int64_t N, int k, float *U, cudaStream_t s);
+int column_cosines_launch(const float *A, const float *B, int D, int k, double *out, cudaStream_t s);
 
 // basis (basis.cu)
 int basis_prepare(const float *Vk, int D, int k, int dtype, void *basis, cudaStream_t s);
 
 // calibration (calibrate.cu)
 size_t calib_workspace_bytes(int D, int k);
+size_t calib_gram_offset();
 int calib_begin(int D, int k, void *ws, cudaStream_t s);
 int calib_accumulate(const void *F, int64_t M, int D, int64_t ld, int dtype, void *ws, cudaStream_t s);
 int calib_finish(int D, int k, float *Vk, double *lambda, double *trace, double *info, void *ws,
