@@ -58,7 +58,7 @@ __global__ void __launch_bounds__(256) left_factors_kernel(const float *C, const
     }
 }
 
-// |<a_j, b_j>| of the unit columns j of two D x k bases (one CTA per column, fixed reduction order)
+// similarity (Fig. 1(b)) of the columns j of two D x k bases (one CTA per column, fixed reduction order)
 __global__ void __launch_bounds__(256) column_cosines_kernel(const float *A, const float *B, int D, int k, double *out) {
     __shared__ double part[256];
     const int j = blockIdx.x;
@@ -78,7 +78,10 @@ __global__ void __launch_bounds__(256) column_cosines_kernel(const float *A, con
         r[q] = part[0];
         __syncthreads();
     }
-    if (threadIdx.x == 0) out[j] = (r[1] > 0.0 && r[2] > 0.0) ? fabs(r[0]) / sqrt(r[1] * r[2]) : 0.0;
+    if (threadIdx.x == 0) {   // cosine similarity (in magnitude: singular vectors are sign-free) x magnitude similarity
+        const double na = sqrt(r[1]), nb = sqrt(r[2]);
+        out[j] = (na > 0.0 && nb > 0.0) ? fabs(r[0]) / (na * nb) * (na < nb ? na / nb : nb / na) : 0.0;
+    }
 }
 
 }  // namespace
