@@ -33,6 +33,10 @@ struct CalibHeader {
     int32_t status;   // SVDCACHE_OK, or the error a kernel of the accumulation recorded
 };
 
+// Width of the iterated block: k wanted columns plus guard columns.  (Half as many guard columns
+// as wanted ones cut the multiplications by G from 36 to 24 at k = 64 on the power-law spectra met
+// here, but the wider Ritz problem cost as much as that saved: 47 -> 46 ms at k = 64, 226 -> 266 ms
+// at k = 128.  A quarter it stays.)
 int ritz_width(int D, int k) {
     int p = std::max(16, k / 4);
     int m = (k + p + 7) / 8 * 8;
@@ -617,7 +621,7 @@ int calib_finish(int D, int k, float *Vk, double *lambda, double *trace, double 
         *z = o[0]; *t = o[1];
     };
 
-    // Every iteration: Z = G Q; Rayleigh-Ritz on span(Q) (S = Q^T Z = W Theta W^T, Q <- Q W,
+    // A Ritz iteration: Z = G Q; Rayleigh-Ritz on span(Q) (S = Q^T Z = W Theta W^T, Q <- Q W,
     // Z <- Z W); residual check; Q <- orthonormalise(Z).  The Ritz rotation keeps the columns
     // of Z close to mutually orthogonal, which is what the scaled Cholesky-QR relies on.
     const double tol = 1e-12;
@@ -631,6 +635,18 @@ int calib_finish(int D, int k, float *Vk, double *lambda, double *trace, double 
         rc = dgemm<double, double, true>(G, D, Q, m, Z, m, D, m, D, false, false, s, ps);   // Z = G Q
         if (rc) return rc;
         ++mult;
+        // The Rayleigh-Ritz step (the m x m eigen-problem is the serial, single-CTA part of an
+        // iteration) runs on the first iterations, which turn the random start block into ordered
+        // eigenvector estimates, and on every fourth one after that; in between the iteration is plain
+        // orthogonal iteration, Q <- orthonormalise(G Q): the QR step takes out of every column its
+        // components along the columns before it, so the columns stay ordered and nearly orthogonal
+        // and the scaled Cholesky-QR stays well conditioned.
+        const bool ritz_step = mult <= 4 || (mult % 4) == 0 || mult == max_mult;
+        if (!ritz_step) {
+            rc = orthonormalize(Z, T, S, X, dead, D, m, (uint64_t)mult + 1, &Q, s, ps);
+            if (rc) return rc;
+            continue;
+        }
         rc = dgemm<double, double, true>(Q, m, Z, m, S, m, m, m, D, false, false, s, ps);   // S = Q^T Z
         if (rc) return rc;
         symmetrize_kernel<<<grid_for((int64_t)m * m), 256, 0, s>>>(S, m, 1);
