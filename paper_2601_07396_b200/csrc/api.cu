@@ -5,6 +5,8 @@
 #include <cstring>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "internal.cuh"
 
 namespace svdc {
@@ -23,6 +25,13 @@ int record_cuda(cudaError_t e) {
 }
 
 int check_last_launch() { return record_cuda(cudaGetLastError()); }
+
+// An NVTX range around an entry point (costs nothing unless a profiler is attached): the kernels
+// of a call show up under its name in a timeline.
+struct NvtxRange {
+    explicit NvtxRange(const char *name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+};
 
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -136,6 +145,7 @@ int svdcache_calibrate_begin(int D, int k, void *ws, size_t bytes, void *stream)
 
 int svdcache_calibrate_accumulate(const void *F, int64_t M, int D, int64_t ld, int dtype, void *ws,
                                   size_t bytes, void *stream) {
+    NvtxRange range("svdcache_calibrate_accumulate");
     if (dtype != SVDCACHE_F32 && dtype != SVDCACHE_BF16) return SVDCACHE_ERR_INVALID_ARG;
     if (M < 0 || D < 8 || D > 16384 || (D % 8) != 0) return SVDCACHE_ERR_BAD_SHAPE;
     if (!ws) return SVDCACHE_ERR_INVALID_ARG;
@@ -151,6 +161,7 @@ int svdcache_calibrate_accumulate(const void *F, int64_t M, int D, int64_t ld, i
 
 int svdcache_calibrate_finish(int D, int k, float *Vk, double *lambda, double *trace, double *info,
                               void *ws, size_t bytes, void *stream) {
+    NvtxRange range("svdcache_calibrate_finish");
     int rc = check_ws(D, k, ws, bytes);
     if (rc) return rc;
     if (!Vk) return SVDCACHE_ERR_INVALID_ARG;
@@ -317,6 +328,7 @@ int svdcache_full_step_batched(int nblocks, const void *F, int64_t ld, size_t F_
                                size_t basis_stride, void *state, size_t state_stride, float *C_out,
                                size_t C_stride, int64_t N, int D, int k, int dtype, float beta,
                                void *stream) {
+    NvtxRange range("svdcache_full_step_batched");
     StepArgs a{};
     a.F = F; a.ld = ld; a.F_stride = F_stride; a.basis = basis; a.basis_stride = basis_stride;
     a.state = state; a.state_stride = state_stride; a.C_out = C_out; a.C_stride = C_stride;
@@ -329,6 +341,7 @@ int svdcache_full_step_batched(int nblocks, const void *F, int64_t ld, size_t F_
 int svdcache_cached_step_batched(int nblocks, const void *state, size_t state_stride, const void *basis,
                                  size_t basis_stride, void *Fhat, int64_t ld, size_t Fhat_stride,
                                  int64_t N, int D, int k, int dtype, int steps_since_full, void *stream) {
+    NvtxRange range("svdcache_cached_step_batched");
     (void)steps_since_full;  // the EMA forecast does not depend on it
     StepArgs a{};
     a.Fhat = Fhat; a.ld = ld; a.Fhat_stride = Fhat_stride; a.basis = basis; a.basis_stride = basis_stride;
@@ -343,6 +356,7 @@ int svdcache_full_step_residual_ema_batched(int nblocks, const void *F, int64_t 
                                             const void *basis, size_t basis_stride, void *state,
                                             size_t state_stride, float *C_out, size_t C_stride, int64_t N,
                                             int D, int k, int dtype, float beta, float beta_r, void *stream) {
+    NvtxRange range("svdcache_full_step_residual_ema_batched");
     if (!(beta_r >= 0.0f && beta_r <= 1.0f)) return SVDCACHE_ERR_INVALID_ARG;
     StepArgs a{};
     a.F = F; a.ld = ld; a.F_stride = F_stride; a.basis = basis; a.basis_stride = basis_stride;
@@ -370,6 +384,7 @@ int svdcache_cached_step_forecast_batched(int nblocks, const void *state, size_t
                                           int64_t N, int D, int k, int dtype, const float *const *C_hist,
                                           size_t C_stride, int predictor, int order, int steps_since_full,
                                           int interval, void *forecast, size_t forecast_stride, void *stream) {
+    NvtxRange range("svdcache_cached_step_forecast_batched");
     StepArgs a{};
     a.Fhat = Fhat; a.ld = ld; a.Fhat_stride = Fhat_stride; a.basis = basis; a.basis_stride = basis_stride;
     a.state = const_cast<void *>(state); a.state_stride = state_stride;
