@@ -561,6 +561,39 @@ def run_sweep(args):
                                           "TFLOPs": round(tf_c, 1), "frac_tensor": round(tf_c / tf_peak, 4)},
                           "peaks": {"hbm_GBps": peak, "bf16_TFLOPs": tf_peak, "source": peak_kind}}), flush=True)
         del state, bases
+    # ---- modes beyond the method's own step (Sec. 4.5, Sec. 5.3), at the FLUX rank: bytes and time per mode ----
+    k = base.k
+    Vk = V_gen[:, :k].float().contiguous()
+    bases = torch.empty(nb, sc.svdcache_basis_bytes(D, k, sc.BF16), dtype=torch.uint8, device=device)
+    for b in range(nb):
+        sc.svdcache_basis_prepare(Vk, sc.BF16, basis=bases[b])
+    state = sc.new_state(N, D, k, sc.BF16, device, blocks=nb)
+    bf, bc = algorithmic_bytes(base, nb)
+    hist = [torch.empty(nb, N, k, dtype=torch.float32, device=device) for _ in range(3)]
+    for h in hist:
+        sc.svdcache_full_step_batched(F, bases, state, k, base.beta, C_out=h)
+    fbuf = torch.empty(nb, sc.svdcache_forecast_bytes(N, k), dtype=torch.uint8, device=device)
+    modes = [
+        ("full step, EMA on the principal part, residual reused (the method)", bf,
+         lambda: sc.svdcache_full_step_batched(F, bases, state, k, base.beta)),
+        ("full step, reuse on both (beta = 0)", bf,
+         lambda: sc.svdcache_full_step_batched(F, bases, state, k, 0.0)),
+        ("full step, EMA on both (beta_R = 0.5; reads the old R as well)", bf + nb * N * D * 2,
+         lambda: sc.svdcache_full_step_residual_ema_batched(F, bases, state, k, base.beta, 0.5)),
+        ("cached step, EMA forecast (the method)", bc,
+         lambda: sc.svdcache_cached_step_batched(state, bases, Fhat, k)),
+    ]
+    for order in (1, 2):
+        modes.append((f"cached step, Newton forecast of order {order} (history read, forecast written, 2 launches)",
+                      bc + nb * N * k * 4 * (order + 1) + nb * N * k * 8,
+                      lambda order=order: sc.svdcache_cached_step_forecast_batched(
+                          state, bases, Fhat, k, hist[:order + 1], sc.PREDICT_NEWTON, 3, base.interval, forecast=fbuf)))
+    for name, nbytes, fn in modes:
+        ms = timed(fn, args.steps)
+        print(json.dumps({"sweep": "mode", "mode": name, "k": k, "blocks": nb, "algorithmic_bytes": nbytes,
+                          "ms": round(ms, 4), "GBps": round(nbytes / ms / 1e6, 1), "frac_hbm": round(nbytes / ms / 1e6 / peak, 4)}),
+              flush=True)
+    del state, bases, hist, fbuf
     del F, Fhat
     torch.cuda.empty_cache()
     k = base.k

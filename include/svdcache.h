@@ -301,8 +301,9 @@ SVDCACHE_API int svdcache_cached_step_forecast_batched(int nblocks, const void *
  *     R <- F - C V_k^T on the first full step, else beta_r R + (1 - beta_r)(F - C V_k^T).
  * beta_r = 0 is svdcache_full_step itself (the method: the residual is reused as it is);
  * beta = beta_r = 0 is "reuse on both" (Eq. 3); beta, beta_r > 0 is "EMA on both".  With
- * beta_r > 0 the step reads the old R as well (N D more elements than the method's step) and
- * runs on the CUDA-core kernels.  Arguments as svdcache_full_step_batched.
+ * beta_r > 0 the step reads the old R as well (N D more elements than the method's step): the
+ * epilogue of the fused kernel loads it and blends before the one rounding to the I/O dtype.
+ * Arguments as svdcache_full_step_batched.
  * ------------------------------------------------------------------------------- */
 SVDCACHE_API int svdcache_full_step_residual_ema_batched(int nblocks, const void *F, int64_t ld,
                                             size_t F_stride, const void *basis, size_t basis_stride,

@@ -53,12 +53,6 @@ static int dispatch(const StepArgs &a_in, bool full, cudaStream_t s) {
     const int want = g_path.load();
     const bool can_umma = umma_supported(a, full);
     if (want == 2 && !can_umma) return SVDCACHE_ERR_BAD_SHAPE;
-    // the residual EMA of the ablation is a read-modify-write of R: it runs on the CUDA-core kernels
-    if (full && a.beta_r > 0.0f) {
-        if (want == 2) return SVDCACHE_ERR_BAD_SHAPE;
-        g_last_path.store(1);
-        return simt_full_step(a, s);
-    }
     const bool use_umma = (want == 2) || (want == 0 && can_umma);
     g_last_path.store(use_umma ? 2 : 1);
     if (use_umma) return full ? umma_full_step(a, s) : umma_cached_step(a, s);

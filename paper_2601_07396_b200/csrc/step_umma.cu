@@ -49,6 +49,8 @@ struct UmmaParams {
     float *C_out;
     size_t C_stride;
     float beta;
+    float beta_r;          // full step: EMA weight of the stored residual (0: the residual is replaced)
+    size_t r_off;          // offset of R in a block's state
 };
 
 struct SmemLayout {
@@ -143,6 +145,23 @@ __device__ __forceinline__ uint4 combine_chunk(uint4 t, const uint32_t *acc) {
         const float r0 = SUBTRACT ? (lo - a0) : (lo + a0);
         const float r1 = SUBTRACT ? (hi - a1) : (hi + a1);
         const __nv_bfloat162 pk = __floats2bfloat162_rn(r0, r1);
+        o[i] = *reinterpret_cast<const uint32_t *>(&pk);
+    }
+    return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+// The same for the residual EMA of the ablation (Sec. 4.5): out = beta_r * old + (1 - beta_r) * (tile - acc),
+// formed in fp32 and rounded once
+__device__ __forceinline__ uint4 combine_chunk_ema(uint4 t, const uint32_t *acc, uint4 old, float beta_r) {
+    const uint32_t w[4] = {t.x, t.y, t.z, t.w}, ow[4] = {old.x, old.y, old.z, old.w};
+    uint32_t o[4];
+    const float omb = 1.0f - beta_r;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
+        const float olo = __uint_as_float(ow[i] << 16), ohi = __uint_as_float(ow[i] & 0xFFFF0000u);
+        const float r0 = lo - __uint_as_float(acc[2 * i]), r1 = hi - __uint_as_float(acc[2 * i + 1]);
+        const __nv_bfloat162 pk = __floats2bfloat162_rn(fmaf(beta_r, olo, omb * r0), fmaf(beta_r, ohi, omb * r1));
         o[i] = *reinterpret_cast<const uint32_t *>(&pk);
     }
     return make_uint4(o[0], o[1], o[2], o[3]);
@@ -530,7 +549,7 @@ __device__ __forceinline__ void stg256(void *dst, uint4 a, uint4 b) {
                  : "memory");
 }
 
-template <bool kTmemA>
+template <bool kTmemA, bool kResEma>
 __global__ void __launch_bounds__(kThreadsFull, 1)
 umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant__ CUtensorMap tm_vt,
                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_rout,
@@ -948,6 +967,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                 SVDC_TRACE_ADD(2, c2);
             }
             // ---- epilogue duty for this group's chunks of pass 2
+            const bool first_unit = kResEma && *(volatile uint32_t *)&header_of(p, un.b)->full_steps == 0;
             const int slab_row0 = un.rt * kTileRows + q * kSlabRows;
             const bool slab_live = (int64_t)slab_row0 < p.N;
             it += CT;   // pass-1 slots are consumed by the MMA warp alone
@@ -966,6 +986,21 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                     if ((it & 1u) != grp) continue;
                     const int c = cg + j;
                     const uint32_t s = fr.idx, ph = fr.ph;
+                    // residual EMA (ablation): this row's 64 columns of the stored R, asked for before the
+                    // waits below so that the loads are under way while the chunk and its accumulator arrive
+                    uint4 r_old[kResEma ? 8 : 1];
+                    bool blend = false;
+                    if constexpr (kResEma) {
+                        const int64_t n = (int64_t)un.rt * kTileRows + row;
+                        blend = !first_unit && n < p.N;
+                        if (blend) {
+                            const uint4 *src = reinterpret_cast<const uint4 *>(p.state + (size_t)un.b * p.state_stride + p.r_off +
+                                                                               ((size_t)n * p.D + (size_t)c * kTileCols) * 2);
+#pragma unroll
+                            for (int cc = 0; cc < 8; ++cc)
+                                r_old[cc] = (c * kTileCols + cc * 8 < p.D) ? __ldcg(src + cc) : make_uint4(0u, 0u, 0u, 0u);
+                        }
+                    }
                     SVDC_TRACE_MARK(e4);
                     if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar.full + 8 * s, ph, abort_flag, 17))) { record_timeout(p, abort_flag, it, ig, ui); goto done; }
                     SVDC_TRACE_ADD(4, e4);
@@ -984,9 +1019,13 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                     __syncwarp();
                     if (lane == 0 && j == last_own) mbar_arrive(bar.acc_empty + 8 * as);   // this warp is done with the group
 #pragma unroll
-                    for (int cc = 0; cc < 8; ++cc)
-                        sts128(tile + (((uint32_t)cc) ^ ((uint32_t)row & 7u)) * 16u,
-                               combine_chunk<true>(t[cc], cc < 4 ? acc0 + cc * 8 : acc1 + (cc - 4) * 8));
+                    for (int cc = 0; cc < 8; ++cc) {
+                        const uint32_t *ac = cc < 4 ? acc0 + cc * 8 : acc1 + (cc - 4) * 8;
+                        uint4 o;
+                        if constexpr (kResEma) o = blend ? combine_chunk_ema(t[cc], ac, r_old[cc], p.beta_r) : combine_chunk<true>(t[cc], ac);
+                        else o = combine_chunk<true>(t[cc], ac);
+                        sts128(tile + (((uint32_t)cc) ^ ((uint32_t)row & 7u)) * 16u, o);
+                    }
                     fence_proxy_async();
                     __syncwarp();
                     if (lane == 0) {
@@ -1135,6 +1174,8 @@ bool fill_params(const StepArgs &a, UmmaParams &p) {
     p.C_out = a.C_out;
     p.C_stride = a.C_stride;
     p.beta = a.beta;
+    p.beta_r = a.beta_r;
+    p.r_off = state_layout(a.N, a.D, a.k, a.dtype).r;
     return true;
 }
 
@@ -1341,15 +1382,18 @@ int umma_full_step(const StepArgs &a, cudaStream_t s) {
     const size_t smem = smem_bytes_full(p);
     const int sms = num_sms();
     const int grid = p.units < sms ? p.units : sms;
-    if (a.k >= 64) {   // operand in tensor memory (fill_full has sized the rings for it)
-        rc = allow_big_smem(umma_full_kernel<true>, kSmemBudget);
-        if (rc) return rc;
-        umma_full_kernel<true><<<grid, kThreadsFull, smem, s>>>(tm_f, tm_vt, tm_v, tm_rout, tm_chat, p);
-    } else {
-        rc = allow_big_smem(umma_full_kernel<false>, kSmemBudget);
-        if (rc) return rc;
-        umma_full_kernel<false><<<grid, kThreadsFull, smem, s>>>(tm_f, tm_vt, tm_v, tm_rout, tm_chat, p);
-    }
+    auto launch = [&](auto kern) {
+        const int rc_attr = allow_big_smem(kern, kSmemBudget);
+        if (rc_attr) return rc_attr;
+        kern<<<grid, kThreadsFull, smem, s>>>(tm_f, tm_vt, tm_v, tm_rout, tm_chat, p);
+        return (int)SVDCACHE_OK;
+    };
+    // operand in tensor memory from k = 64 on (fill_full has sized the rings for it); the residual EMA
+    // of the ablation is an instantiation of its own (its old-R loads cost registers)
+    const bool ema = a.beta_r > 0.0f;
+    if (a.k >= 64) rc = ema ? launch(umma_full_kernel<true, true>) : launch(umma_full_kernel<true, false>);
+    else rc = ema ? launch(umma_full_kernel<false, true>) : launch(umma_full_kernel<false, false>);
+    if (rc) return rc;
     count_launch();
     return check_last_launch();
 }

@@ -126,7 +126,8 @@ def test_forecast_batched_equals_per_block():
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("N,D,k,dtype", [(256, 1152, 32, "f32"), (300, 1024, 64, "bf16"), (129, 3072, 128, "bf16")])
+@pytest.mark.parametrize("N,D,k,dtype", [(256, 1152, 32, "f32"), (300, 1024, 64, "bf16"), (129, 3072, 128, "bf16"),
+                                         (515, 1000, 32, "bf16"), (2000, 512, 16, "bf16")])
 def test_residual_ema_full_step(N, D, k, dtype):
     """The ablation's full step: Chat as in the method, the stored residual an EMA of the residuals;
     then the cached step on that state."""
@@ -145,7 +146,7 @@ def test_residual_ema_full_step(N, D, k, dtype):
         F = st.features(t)
         C = torch.empty(N, k, dtype=torch.float32, device=DEV)
         sc.svdcache_full_step_residual_ema_batched(F, basis, state, k, beta, beta_r, C_out=C)
-        assert sc.svdcache_last_path() == 1
+        assert sc.svdcache_last_path() == (1 if dtype == "f32" else 2)   # bf16: the tensor-core full step blends in its epilogue
         sc.svdcache_cached_step(state, basis, Fhat, k)
         Fh = _np(F)
         Cr, rhat, chat = oracle.full_step_residual_ema(Fh, V, float(np.float32(beta)), float(np.float32(beta_r)), chat, rhat)
