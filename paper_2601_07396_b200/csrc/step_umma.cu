@@ -41,7 +41,8 @@ struct UmmaParams {
     int stages, a_bufs;
     uint32_t a_half_bytes, a_bytes;
     int gc, acc_stages, acc_cols, v_slots;   // chunks per MMA group, TMEM ring, basis ring
-    int dual, acc_stride;                    // cached step: separate hi / lo accumulators; TMEM columns per ring stage
+    int acc_stride;                          // TMEM columns per stage of the accumulator ring
+    int acc_base;                            // cached step: first TMEM column of the accumulator ring (operand buffers before it)
     uint32_t vslice_bytes;
     uint32_t a_region_bytes, chat_stage_off; // full step: A operand (+ Chat staging when it is not in place)
     char *state;
@@ -203,23 +204,33 @@ __device__ __forceinline__ int last_own_chunk(uint32_t it0, int nsub, uint32_t g
 // Cached step (Sec. 3.5):  Fhat = Chat V_k^T + R
 //
 // A unit is one 128-row tile of one block (times a column range when the launch is too
-// small to occupy the GPU otherwise).  Its A operand -- the split-bf16 copy of Chat that the
-// full step left in the state -- arrives by TMA.  The columns are walked in groups of
+// small to occupy the GPU otherwise).  Its A operand is the split-bf16 copy of Chat that the
+// full step left in the state (or a forecast of it).  The columns are walked in groups of
 // `gc` 64-column chunks: one basis slice (gc*64 x k) per group feeds MMAs of N = gc*64
-// (few, wide instructions: a dependent MMA costs ~200 cycles whatever its N), while the R
-// tiles of the group's chunks stream through their own ring and meet the accumulator in
+// (few, wide instructions: an MMA of M = 128, K = 16 costs ~105 cycles up to N = 128), while the
+// R tiles of the group's chunks stream through their own ring and meet the accumulator in
 // the epilogue.
 //
-// Warp roles (320 threads): 0 = TMA producer (lane 0: R tiles and basis slices, lane 1: A tiles),
-// 1 = MMA issuer (+ TMEM owner), 2..9 = two
-// epilogue groups of four warps (TMEM lane quarter = warp % 4; group g takes the chunks
-// whose running index is g modulo 2).  Each epilogue warp owns a 32-row slab of the chunk
-// from the TMEM read to its own TMA store, so the eight warps never meet at a barrier.
+// Where the operand lives:
+//   k <= 64   two shared-memory buffers (32 KB each at k = 64), filled by TMA one unit ahead;
+//   k >= 128  tensor memory (kTmemA).  The tile's 2 * nkb pieces (hi and lo words of every 64-wide K
+//     block, 16 KB each) travel through the R ring like any chunk, one unit ahead of their use;
+//     the epilogue warps move them into TMEM (128 bytes of a row = 32 columns, two bf16 each) and
+//     the MMAs take their A operand from there.  TMEM columns: a_bufs * k of operand (two buffers
+//     at k = 128, one above), then the accumulator ring.  All of shared memory goes to the rings.
+//
+// Warp roles (320 threads): 0 = TMA producer (lane 0: R tiles and basis slices -- and the operand
+// pieces when they go through the ring --, lane 1: operand tiles for the shared-memory buffers),
+// 1 = MMA issuer (+ TMEM owner), 2..9 = two epilogue groups of four warps (TMEM lane quarter =
+// warp % 4; group g takes the chunks whose running index is g modulo 2).  Each epilogue warp owns a
+// 32-row slab of the chunk from the TMEM read to its own TMA store, so the eight warps never meet
+// at a barrier.
 // ======================================================================================
 constexpr int kThreadsCached = 320;
 constexpr int kSlabRows = 32;                              // rows one epilogue warp stores
 constexpr uint32_t kSlabBytes = kSlabRows * kTileCols * 2; // 4 KB
 
+template <bool kTmemA>
 __global__ void __launch_bounds__(kThreadsCached, 1)
 umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_constant__ CUtensorMap tm_v,
                    const __grid_constant__ CUtensorMap tm_ahi, const __grid_constant__ CUtensorMap tm_alo,
@@ -227,7 +238,7 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t a_base0 = base;
-    const uint32_t v_base0 = a_base0 + (uint32_t)p.a_bufs * p.a_bytes;
+    const uint32_t v_base0 = a_base0 + (kTmemA ? 0u : (uint32_t)p.a_bufs * p.a_bytes);
     const uint32_t stage0 = v_base0 + (uint32_t)p.v_slots * p.vslice_bytes;
     const Bars bar = bars_at(stage0 + (uint32_t)p.stages * kTileBytes);
     uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
@@ -237,13 +248,28 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     SVDC_TRACE_DECL
     const uint32_t tmem_cols = 512;
+    // kTmemA (k >= 128): the operand tile travels through the R ring as 2 * nkb ordinary chunks
+    // (hi and lo part of every 64-wide K block) and the epilogue warps copy it into tensor memory
+    const int n_a_chunks = 2 * p.nkb;
+    // units this CTA works on: those of blocks that have seen a full step
+    auto next_live = [&](int u) {
+        while (u < p.units && *(volatile uint32_t *)&header_of(p, decode_unit(p, u).b)->full_steps == 0) u += (int)gridDim.x;
+        return u;
+    };
+    // the operand of the next unit is requested, and copied, right before the R chunks of this group
+    // of the current one: the first with two operand buffers, the last with one (its MMAs, the last
+    // readers of the buffer, have their basis slice requested by then)
+    auto insert_group = [&](const Unit &un) { return p.a_bufs > 1 ? 0 : (un.c1 - un.c0 + p.gc - 1) / p.gc - 1; };
 
     if (threadIdx.x == 0) {
         // R slot: free again once the four slab stores have read it.  Accumulator: one arrival
         // from each of the eight epilogue warps per group (see group_share below).
         for (int s = 0; s < p.stages; ++s) { mbar_init(bar.full + 8 * s, 1); mbar_init(bar.empty + 8 * s, 4); }
         for (int s = 0; s < p.acc_stages; ++s) { mbar_init(bar.acc_full + 8 * s, 1); mbar_init(bar.acc_empty + 8 * s, 8); }
-        for (int s = 0; s < p.a_bufs; ++s) { mbar_init(bar.a_full + 8 * s, 1); mbar_init(bar.a_empty + 8 * s, 1); }
+        for (int s = 0; s < p.a_bufs; ++s) {   // operand in TMEM: four warps announce each of its chunks
+            mbar_init(bar.a_full + 8 * s, kTmemA ? 4u * (uint32_t)n_a_chunks : 1u);
+            mbar_init(bar.a_empty + 8 * s, 1);
+        }
         for (int s = 0; s < p.v_slots; ++s) { mbar_init(bar.v_full + 8 * s, 1); mbar_init(bar.v_empty + 8 * s, 1); }
         *abort_flag = 0;
         fence_barrier_init();
@@ -264,11 +290,9 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer ---
-        // The A tile of live unit number ua (of unit ux): with two operand buffers (k <= 64) the
-        // requests run on a lane of their own, one unit ahead of the MMAs, and never hold up the R
-        // and basis streams (+4 % on the FLUX shape); with a single buffer the tile can only be
-        // requested when the MMAs of the unit before are done, and it goes first, in order, on the
-        // stream lane -- R tiles requested ahead of it only delay it (measured at k = 128).
+        // Operand in shared memory (k <= 64, two buffers): the A tile of live unit number ua (of unit
+        // ux) is requested on a lane of its own, one unit ahead of the MMAs, and never holds up the R
+        // and basis streams (+4 % on the FLUX shape).
         auto request_a = [&](const Unit &ux, uint32_t ua) {
             const uint32_t ab = ua % p.a_bufs;
             SVDC_TRACE_MARK(p0);
@@ -284,18 +308,75 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
             }
             return true;
         };
+        if constexpr (kTmemA) {
+            if (lane == 0) {
+                RingPos fr, vr;                        // next ring slot, next basis slot
+                auto mark_dead = [&](int u0, int u1) {   // blocks without a full step: report once per block
+                    for (int u = u0; u < u1 && u < p.units; u += (int)gridDim.x) {
+                        const Unit x = decode_unit(p, u);
+                        if (x.rt == 0 && x.c0 == 0 && *(volatile uint32_t *)&header_of(p, x.b)->full_steps == 0)
+                            header_of(p, x.b)->status = SVDCACHE_ERR_STATE;
+                    }
+                };
+                auto request_a_chunks = [&](const Unit &ux) {   // hi K block 0, lo K block 0, hi K block 1, ...
+                    for (int i = 0; i < n_a_chunks; ++i) {
+                        const uint32_t s = fr.idx;
+                        SVDC_TRACE_MARK(p0);
+                        if (!mbar_wait(bar.empty + 8 * s, fr.ph ^ 1u, abort_flag, 1)) return false;
+                        SVDC_TRACE_ADD(0, p0);
+                        fr.step((uint32_t)p.stages);
+                        mbar_arrive_expect_tx(bar.full + 8 * s, kTileBytes);
+                        tma_load_3d(stage0 + s * kTileBytes, (i & 1) ? &tm_alo : &tm_ahi, bar.full + 8 * s,
+                                    (i >> 1) * p.kb_elems, ux.rt * kTileRows, ux.b);
+                    }
+                    return true;
+                };
+                int u = next_live((int)blockIdx.x);
+                mark_dead((int)blockIdx.x, u);
+                if (u < p.units && !request_a_chunks(decode_unit(p, u))) { record_timeout(p, abort_flag); goto done; }
+                while (u < p.units) {
+                    const Unit un = decode_unit(p, u);
+                    const int u_next = next_live(u + (int)gridDim.x);
+                    mark_dead(u + (int)gridDim.x, u_next);
+                    const int g_ins = insert_group(un);
+                    int g = 0;
+                    for (int cg = un.c0; cg < un.c1; cg += p.gc, ++g) {
+                        const uint32_t vs = vr.idx;
+                        SVDC_TRACE_MARK(p1);
+                        if (!mbar_wait(bar.v_empty + 8 * vs, vr.ph ^ 1u, abort_flag, 2)) { record_timeout(p, abort_flag); goto done; }
+                        SVDC_TRACE_ADD(1, p1);
+                        vr.step((uint32_t)p.v_slots);
+                        const uint32_t vdst = v_base0 + vs * p.vslice_bytes;
+                        mbar_arrive_expect_tx(bar.v_full + 8 * vs, p.vslice_bytes);
+                        for (int kb = 0; kb < p.nkb; ++kb)
+                            tma_load_3d(vdst + kb * (p.gc * kTileCols * p.kb_bytes), &tm_v, bar.v_full + 8 * vs,
+                                        kb * p.kb_elems, cg * kTileCols, un.b);
+                        if (g == g_ins && u_next < p.units && !request_a_chunks(decode_unit(p, u_next))) {
+                            record_timeout(p, abort_flag);
+                            goto done;
+                        }
+                        const int ce = min(cg + p.gc, un.c1);
+                        for (int c = cg; c < ce; ++c) {
+                            const uint32_t s = fr.idx;
+                            SVDC_TRACE_MARK(p2);
+                            if (!mbar_wait(bar.empty + 8 * s, fr.ph ^ 1u, abort_flag, 3)) { record_timeout(p, abort_flag); goto done; }
+                            SVDC_TRACE_ADD(2, p2);
+                            fr.step((uint32_t)p.stages);
+                            mbar_arrive_expect_tx(bar.full + 8 * s, kTileBytes);
+                            tma_load_3d(stage0 + s * kTileBytes, &tm_r, bar.full + 8 * s, c * kTileCols, un.rt * kTileRows, un.b);
+                        }
+                    }
+                    u = u_next;
+                }
+            }
+        } else
         if (lane == 0) {
             RingPos fr, vr;                            // next R slot, next basis slot
-            uint32_t ua = 0;
             for (int u = blockIdx.x; u < p.units; u += gridDim.x) {
                 const Unit un = decode_unit(p, u);
                 if (*(volatile uint32_t *)&header_of(p, un.b)->full_steps == 0) {
                     if (un.rt == 0 && un.c0 == 0) header_of(p, un.b)->status = SVDCACHE_ERR_STATE;
                     continue;
-                }
-                if (p.a_bufs == 1) {
-                    if (!request_a(un, ua)) { record_timeout(p, abort_flag); goto done; }
-                    ++ua;
                 }
                 for (int cg = un.c0; cg < un.c1; cg += p.gc) {
                     const uint32_t vs = vr.idx;
@@ -320,7 +401,7 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
                     }
                 }
             }
-        } else if (lane == 1 && p.a_bufs > 1) {
+        } else if (lane == 1) {
             uint32_t ua = 0;
             for (int u = blockIdx.x; u < p.units; u += gridDim.x) {
                 const Unit ux = decode_unit(p, u);
@@ -342,6 +423,7 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
                 SVDC_TRACE_MARK(m0);
                 if (!mbar_wait(bar.a_full + 8 * ab, (ui / p.a_bufs) & 1u, abort_flag, 4)) { record_timeout(p, abort_flag); goto done; }
                 SVDC_TRACE_ADD(0, m0);
+                if constexpr (kTmemA) tc_fence_after();   // the operand was written by tcgen05.st of other threads
                 const uint64_t a_desc0 = smem_desc_kmajor(a_base0 + ab * p.a_bytes, p.kb_bytes);
                 for (int cg = un.c0; cg < un.c1; cg += p.gc) {
                     const uint32_t vs = vr.idx, as = ar.idx;
@@ -357,24 +439,21 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
                     tc_fence_after();
                     SVDC_TRACE_MARK(m3);
                     const uint32_t idesc = idesc_bf16(kTileRows, nsub * kTileCols);
-                    const uint32_t d_tmem = tmem_base + as * p.acc_stride;
+                    const uint32_t d_tmem = tmem_base + (uint32_t)p.acc_base + as * p.acc_stride;
                     const uint64_t v_desc0 = smem_desc_kmajor(v_base0 + vs * p.vslice_bytes, p.kb_bytes);
-                    if (p.dual) {
-                        // Narrow groups (N <= 128) leave a dependent MMA chain latency-bound: the hi and the
-                        // lo part of the operand go to accumulators of their own, issued alternately, and
-                        // the epilogue adds the two.
-                        const uint32_t d_lo = d_tmem + p.acc_cols;
+                    if constexpr (kTmemA) {
+                        // operand buffer ab: k/2 columns of hi words, then k/2 of lo words (two bf16 per
+                        // 32-bit column); one K step of 16 is 8 columns
+                        const uint32_t a_t = tmem_base + ab * (uint32_t)p.k;
                         uint32_t acc = 0;
-                        for (int kb = 0; kb < p.nkb; ++kb) {
-                            const uint64_t a_hi = a_desc0 + ((kb * (kTileRows * p.kb_bytes)) >> 4);
-                            const uint64_t a_lo = a_hi + (p.a_half_bytes >> 4);
-                            const uint64_t v_kb = v_desc0 + ((kb * (p.gc * kTileCols * p.kb_bytes)) >> 4);
-                            for (int ks = 0; ks < ksteps; ++ks) {
-                                mma_bf16_ss(d_tmem, a_hi + 2 * ks, v_kb + 2 * ks, idesc, acc);
-                                mma_bf16_ss(d_lo, a_lo + 2 * ks, v_kb + 2 * ks, idesc, acc);
-                                acc = 1;
+                        for (int part = 0; part < 2; ++part)
+                            for (int kb = 0; kb < p.nkb; ++kb) {
+                                const uint64_t v_kb = v_desc0 + ((kb * (p.gc * kTileCols * p.kb_bytes)) >> 4);
+                                for (int ks = 0; ks < ksteps; ++ks) {
+                                    mma_bf16_ts(d_tmem, a_t + (uint32_t)(part * (p.k >> 1) + kb * 32 + ks * 8), v_kb + 2 * ks, idesc, acc);
+                                    acc = 1;
+                                }
                             }
-                        }
                     } else {
                         uint32_t acc = 0;
                         for (int part = 0; part < 2; ++part)
@@ -400,14 +479,59 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
         // ---------------------------------------------------------------- epilogue ---
         const int q = warp & 3, row = q * kSlabRows + lane;
         const uint32_t grp = (uint32_t)(warp - 2) >> 2;
-        uint32_t it = 0;
+        uint32_t it = 0, ua = 0;   // chunks taken from the ring, live units begun
         RingPos fr, ar;   // R slot of chunk `it`, accumulator stage of the next group
+        // kTmemA: the operand chunks of live unit number `n` leave the ring for TMEM buffer n % a_bufs.
+        // Every warp waits for the buffer's release (the MMAs of its last user have completed), each
+        // in its turn, so no phase of that barrier goes unseen; a chunk is taken by the group its
+        // running index selects, like an R chunk, and each of the four warps moves the 32 rows of its
+        // TMEM lane quarter: 128 bytes of a row are 32 columns.
+        auto copy_operand = [&](uint32_t n) {
+            const uint32_t ab = n % (uint32_t)p.a_bufs;
+            SVDC_TRACE_MARK(e4);
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar.a_empty + 8 * ab, ((n / (uint32_t)p.a_bufs) & 1u) ^ 1u, abort_flag, 11)))
+                return false;
+            SVDC_TRACE_ADD(4, e4);
+            tc_fence_after();
+            for (int i = 0; i < n_a_chunks; ++i, ++it, fr.step((uint32_t)p.stages)) {
+                if ((it & 1u) != grp) continue;
+                const uint32_t s = fr.idx;
+                SVDC_TRACE_MARK(e5);
+                if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar.full + 8 * s, fr.ph, abort_flag, 12))) return false;
+                SVDC_TRACE_ADD(5, e5);
+                const uint32_t tile = stage0 + s * kTileBytes + (uint32_t)row * 128u;
+                uint32_t w[32];
+#pragma unroll
+                for (int cc = 0; cc < 8; ++cc) {
+                    const uint4 t = lds128(tile + (((uint32_t)cc) ^ ((uint32_t)row & 7u)) * 16u);
+                    w[4 * cc] = t.x; w[4 * cc + 1] = t.y; w[4 * cc + 2] = t.z; w[4 * cc + 3] = t.w;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar.empty + 8 * s);
+                tmem_st_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + ab * (uint32_t)p.k +
+                                  (uint32_t)((i & 1) * (p.k >> 1) + (i >> 1) * 32), w);
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar.a_full + 8 * ab);
+            }
+            return true;
+        };
+        if constexpr (kTmemA) {
+            if (next_live((int)blockIdx.x) < p.units && !copy_operand(0)) { record_timeout(p, abort_flag); goto done; }
+        }
         for (int u = blockIdx.x; u < p.units; u += gridDim.x) {
             const Unit un = decode_unit(p, u);
             if (*(volatile uint32_t *)&header_of(p, un.b)->full_steps == 0) continue;
             const int slab_row0 = un.rt * kTileRows + q * kSlabRows;
             const bool slab_live = (int64_t)slab_row0 < p.N;
-            for (int cg = un.c0; cg < un.c1; cg += p.gc) {
+            const bool more = kTmemA && next_live(u + (int)gridDim.x) < p.units;
+            const int g_ins = insert_group(un);
+            ++ua;
+            for (int cg = un.c0, g = 0; cg < un.c1; cg += p.gc, ++g) {
+                if constexpr (kTmemA) {
+                    if (g == g_ins && more && !copy_operand(ua)) { record_timeout(p, abort_flag); goto done; }
+                }
                 const uint32_t as = ar.idx, aph = ar.ph;
                 ar.step((uint32_t)p.acc_stages);
                 const int nsub = min(p.gc, un.c1 - cg);
@@ -426,24 +550,13 @@ umma_cached_kernel(const __grid_constant__ CUtensorMap tm_r, const __grid_consta
                     SVDC_TRACE_MARK(e2);
                     tc_fence_after();
                     const uint32_t tile = stage0 + s * kTileBytes + (uint32_t)row * 128u;
-                    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + as * p.acc_stride + j * kTileCols;
+                    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)p.acc_base + as * p.acc_stride + j * kTileCols;
                     uint32_t acc0[32], acc1[32];
                     tmem_ld_32x32(taddr, acc0);
                     tmem_ld_32x32(taddr + 32, acc1);
                     uint4 t[8];
 #pragma unroll
                     for (int cc = 0; cc < 8; ++cc) t[cc] = lds128(tile + (((uint32_t)cc) ^ ((uint32_t)row & 7u)) * 16u);
-                    if (p.dual) {   // product = hi-part accumulator + lo-part accumulator
-                        uint32_t lo0[32], lo1[32];
-                        tmem_ld_32x32(taddr + p.acc_cols, lo0);
-                        tmem_ld_32x32(taddr + p.acc_cols + 32, lo1);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            acc0[i] = __float_as_uint(__uint_as_float(acc0[i]) + __uint_as_float(lo0[i]));
-                            acc1[i] = __float_as_uint(__uint_as_float(acc1[i]) + __uint_as_float(lo1[i]));
-                        }
-                    }
                     tmem_wait_ld();
                     tc_fence_before();
                     __syncwarp();
@@ -1235,24 +1348,53 @@ size_t smem_bytes_full(const UmmaParams &p) {
            kBarBytes + 64;
 }
 
+// From k = 128 on the cached step keeps its operand in tensor memory (the kernel's kTmemA): one tile
+// of the split pair would take 64 KB of shared memory and more, which left room for a single
+// buffer -- a bubble at every unit boundary -- and a short R ring (measured at k = 128 / 256 on FLUX
+// rows: 0.75 / 0.38 of the copy bandwidth with the operand in shared memory, 0.83-0.91 / 0.64 so).
+// TMEM bounds the rank: k columns of operand and two accumulators.
+bool cached_operand_in_tmem(int k) { return k >= 128 && k + 2 * kTileCols <= 512; }
+
 bool fill_cached(const StepArgs &a, UmmaParams &p) {
     if (!fill_params(a, p)) return false;
     fill_groups(a, p);
-    p.dual = p.gc <= 2 ? 1 : 0;
-    p.acc_stride = p.acc_cols * (p.dual ? 2 : 1);
-    p.acc_stages = 512 / p.acc_stride < kAccStages ? 512 / p.acc_stride : kAccStages;
     const size_t avail = kSmemBudget - 1024 /*alignment*/ - kBarBytes - 64;
+    if (cached_operand_in_tmem(a.k)) {
+        // TMEM: operand buffers of k columns first (two while two accumulators still fit behind
+        // them), then the accumulator ring.  Groups of two chunks while they fit: N = 128 is the
+        // narrowest MMA that costs no more than a narrower one.
+        p.gc = a.k + 2 * 2 * kTileCols <= 512 ? 2 : 1;
+        p.acc_cols = p.gc * kTileCols;
+        p.acc_stride = p.acc_cols;
+        p.a_bufs = 2 * a.k + 2 * p.acc_cols <= 512 ? 2 : 1;
+        p.acc_base = p.a_bufs * a.k;
+        p.acc_stages = (512 - p.acc_base) / p.acc_stride < kAccStages ? (512 - p.acc_base) / p.acc_stride : kAccStages;
+        p.vslice_bytes = (uint32_t)p.gc * kTileCols * a.k * 2;
+        auto stages_for = [&](int v_slots) {
+            const size_t fixed = (size_t)v_slots * p.vslice_bytes;
+            if (fixed + 4 * (size_t)kTileBytes > avail) return 0;
+            int st = (int)((avail - fixed) / kTileBytes);
+            if (st > kMaxStages) st = kMaxStages;
+            return st & ~1;   // even: a slot then always serves the same epilogue group (chunk parity)
+        };
+        p.v_slots = stages_for(3) >= 8 ? 3 : 2;
+        p.stages = stages_for(p.v_slots);
+        return p.stages >= 4 && p.acc_stages >= 2;
+    }
+    // operand in shared memory, two buffers (k <= 64)
+    p.acc_base = 0;
+    p.acc_stride = p.acc_cols;
     const size_t fixed = (size_t)p.v_slots * p.vslice_bytes;
-    p.a_bufs = (2 * (size_t)p.a_bytes + fixed + 6 * (size_t)kTileBytes <= avail) ? 2 : 1;
-    if ((size_t)p.a_bufs * p.a_bytes + fixed + 2 * (size_t)kTileBytes > avail) return false;
-    p.stages = (int)((avail - (size_t)p.a_bufs * p.a_bytes - fixed) / kTileBytes);
+    p.a_bufs = 2;
+    if (2 * (size_t)p.a_bytes + fixed + 6 * (size_t)kTileBytes > avail) return false;
+    p.stages = (int)((avail - 2 * (size_t)p.a_bytes - fixed) / kTileBytes);
     if (p.stages > kMaxStages) p.stages = kMaxStages;
     p.stages &= ~1;   // even: a slot then always serves the same epilogue group (chunk parity)
     return true;
 }
 size_t smem_bytes_cached(const UmmaParams &p) {
-    return 1024 + (size_t)p.a_bufs * p.a_bytes + (size_t)p.v_slots * p.vslice_bytes + (size_t)p.stages * kTileBytes +
-           kBarBytes + 64;
+    const size_t a_smem = cached_operand_in_tmem(p.k) ? 0 : (size_t)p.a_bufs * p.a_bytes;
+    return 1024 + a_smem + (size_t)p.v_slots * p.vslice_bytes + (size_t)p.stages * kTileBytes + kBarBytes + 64;
 }
 
 bool shape_ok(const StepArgs &a) {
@@ -1283,16 +1425,16 @@ int umma_cached_step(const StepArgs &a, cudaStream_t s) {
     if (!fill_cached(a, p)) return SVDCACHE_ERR_BAD_SHAPE;
     // Units: a row tile, or a column range of it (in whole MMA groups).  The split is the one that
     // minimises what the busiest CTA has to stream, in chunks of R + Fhat traffic (32 KB) -- and,
-    // among splits within 2 % of that, the finest when the operand is double-buffered: CTAs that
+    // among splits within a few per cent of that, the finest one the operand buffers allow: CTAs that
     // work on neighbouring column ranges of the same rows at the same time read and write whole
     // DRAM pages together (measured on the FLUX shape: 6.3 TB/s with single-group units, 5.7 with
-    // whole tiles).  With a single operand buffer (k >= 128) every unit waits for its own copy of
-    // the tile's A operand with empty rings (~4 chunks' worth, plus the a_bytes it re-reads), which
-    // outweighs that: 5.7 TB/s with whole tiles at k = 128, 4.2 with single-group units.
+    // whole tiles).  Every unit fetches its own copy of the tile's operand; with the operand in
+    // tensor memory that is nkb chunks' worth of traffic per unit, which the count includes.
     const int sms = num_sms();
     const int tiles = p.row_tiles * a.nblocks;
     const int groups_total = (p.chunks_total + p.gc - 1) / p.gc;
-    const int unit_cost = p.a_bufs == 1 ? (int)((p.a_bytes + 2 * kTileBytes - 1) / (2 * kTileBytes)) + 4 : 0;
+    const bool a_tmem = cached_operand_in_tmem(a.k);
+    const int unit_cost = a_tmem ? p.nkb : 0;
     auto load_of = [&](int ds, int *eff_out, int *gps_out) {
         const int gps = (groups_total + ds - 1) / ds;            // groups per slice
         const int eff = (groups_total + gps - 1) / gps;          // slices that result
@@ -1311,7 +1453,8 @@ int umma_cached_step(const StepArgs &a, cudaStream_t s) {
     if (p.a_bufs > 1)
         for (int ds = 1; ds <= groups_total && ds <= 16; ++ds) {
             int eff, gps;
-            if (load_of(ds, &eff, &gps) * 50 <= best_load * 51 && eff > p.dsplit) { p.dsplit = eff; p.chunks_per_slice = gps * p.gc; }
+            const int slack = a_tmem ? 20 : 50;   // within 5 % (operand in tensor memory: measured at k = 128), else 2 %
+            if (load_of(ds, &eff, &gps) * slack <= best_load * (slack + 1) && eff > p.dsplit) { p.dsplit = eff; p.chunks_per_slice = gps * p.gc; }
         }
     p.units = tiles * p.dsplit;
 
@@ -1337,10 +1480,16 @@ int umma_cached_step(const StepArgs &a, cudaStream_t s) {
     if (rc) return rc;
 
     const size_t smem = smem_bytes_cached(p);
-    rc = allow_big_smem(umma_cached_kernel, kSmemBudget);
-    if (rc) return rc;
     const int grid = p.units < sms ? p.units : sms;
-    umma_cached_kernel<<<grid, kThreadsCached, smem, s>>>(tm_r, tm_v, tm_ahi, tm_alo, tm_out, p);
+    if (a_tmem) {
+        rc = allow_big_smem(umma_cached_kernel<true>, kSmemBudget);
+        if (rc) return rc;
+        umma_cached_kernel<true><<<grid, kThreadsCached, smem, s>>>(tm_r, tm_v, tm_ahi, tm_alo, tm_out, p);
+    } else {
+        rc = allow_big_smem(umma_cached_kernel<false>, kSmemBudget);
+        if (rc) return rc;
+        umma_cached_kernel<false><<<grid, kThreadsCached, smem, s>>>(tm_r, tm_v, tm_ahi, tm_alo, tm_out, p);
+    }
     count_launch();
     return check_last_launch();
 }

@@ -135,20 +135,21 @@ def test_first_full_step_never_reads_the_old_state(D):
     _play(spec, 0, None, range(3), path=2, poison=True, sample=streams.sample_rows(20000, 4096, tile=128))
 
 
-@pytest.mark.parametrize("path,rows,D", [(0, 200, 512), (2, 200, 512), (2, 700, 3072)])
-def test_batched_equals_per_block_and_oracle(path, rows, D):
+@pytest.mark.parametrize("path,rows,D,k", [(0, 200, 512, 64), (2, 200, 512, 64), (2, 700, 3072, 64),
+                                          (2, 700, 3072, 128), (2, 300, 1024, 256)])
+def test_batched_equals_per_block_and_oracle(path, rows, D, k):
     """One batched launch over three blocks (tiles run across block boundaries) against three
     per-block launches (bitwise) and the oracle."""
     prev = sc.svdcache_set_path(path)
     try:
-        _batched_case(rows, D)
+        _batched_case(rows, D, k)
     finally:
         sc.svdcache_set_path(prev)
 
 
-def _batched_case(rows, D):
-    spec = streams.StreamSpec("batch", blocks=3, rows=rows, D=D, dtype="bf16", k=64, T=4, interval=2,
-                              rank=128, amp=30.0, power=1.0, noise_std=0.02)
+def _batched_case(rows, D, k=64):
+    spec = streams.StreamSpec("batch", blocks=3, rows=rows, D=D, dtype="bf16", k=k, T=4, interval=2,
+                              rank=2 * k, amp=30.0, power=1.0, noise_std=0.02)
     nb, N, D, k, dt = 3, spec.rows, spec.D, spec.k, sc.BF16
     bases = torch.stack([sc.svdcache_basis_prepare(
         streams.BlockStream(spec, b, device=DEV).V_gen[:, :k].float().contiguous(), dt) for b in range(nb)])
@@ -279,6 +280,33 @@ def test_cached_step_before_any_full_step_is_reported_not_computed():
     # reset clears the sticky status
     sc.svdcache_state_reset(state, N, D, k, dt)
     assert sc.svdcache_state_query(state) == (0, 0)
+
+
+@pytest.mark.parametrize("k", [64, 128, 256])
+def test_batched_cached_step_skips_blocks_without_a_full_step(k):
+    """A batch in which only some blocks have seen a full step: those are reconstructed exactly as
+    by a call of their own, the others are reported (status -4) and their output is left alone --
+    at every rank the operand reaches the tensor cores by a different route."""
+    N, D, dt, nb = 900, 1024, sc.BF16, 4
+    spec = streams.StreamSpec("mixed", blocks=nb, rows=N, D=D, dtype="bf16", k=k, T=2, interval=1,
+                              rank=2 * k, amp=30.0, power=1.0, noise_std=0.02)
+    bases = torch.stack([sc.svdcache_basis_prepare(
+        streams.BlockStream(spec, b, device=DEV).V_gen[:, :k].float().contiguous(), dt) for b in range(nb)])
+    state = sc.new_state(N, D, k, dt, DEV, blocks=nb)
+    live = (0, 2)
+    for b in live:
+        sc.svdcache_full_step(streams.BlockStream(spec, b, device=DEV).features(0), bases[b], state[b], k, 0.9)
+    out = torch.full((nb, N, D), 7.0, dtype=torch.bfloat16, device=DEV)
+    sc.svdcache_cached_step_batched(state, bases, out, k)
+    ref = torch.empty(N, D, dtype=torch.bfloat16, device=DEV)
+    for b in range(nb):
+        if b in live:
+            sc.svdcache_cached_step(state[b], bases[b], ref, k)
+            assert torch.equal(out[b], ref)
+            assert sc.svdcache_state_query(state[b]) == (1, 0)
+        else:
+            assert bool((out[b] == 7.0).all())
+            assert sc.svdcache_state_query(state[b]) == (0, -4)
 
 
 def test_beta_zero_returns_the_last_full_feature():
