@@ -4,10 +4,11 @@
 //   V_k = top-k eigenvectors of G      block subspace iteration with Rayleigh-Ritz:
 //        Z = G Q;  S = Q^T Z;  S = W Theta W^T (parallel cyclic Jacobi);  Q <- Q W;
 //        stop when |G v - theta v| <= tol * theta_1 for the k leading pairs;
-//        else Q <- orthonormalise(Z) (Cholesky-QR, applied twice) and repeat.
+//        else Q <- orthonormalise(p(G) Q) (Cholesky-QR, applied twice) and repeat, p a Chebyshev
+//        polynomial of degree 1 or 2 that damps the spectrum below the block's smallest Ritz value.
 //
 // Everything runs on the device in fp64 on the plain ALUs; the host only sequences
-// launches and reads one convergence number per Rayleigh-Ritz step.  The eigen-gap at k
+// launches and reads two numbers per Rayleigh-Ritz step (residual, filter degree).  The eigen-gap at k
 // of the power-law spectra met here is ~1e-6 of the leading eigenvalue, so fp32
 // anywhere in this path would miss a 1e-4 bound on the principal-angle cosines.
 #include <algorithm>
@@ -332,6 +333,82 @@ __global__ void __launch_bounds__(1024) chol_inv_kernel(double *S, double *XT, i
 // Indexing: XT[c][i] holds X[i][c] = (L^-1)[i][c], i.e. (L^-T)[c][i]; the product Z XT
 // reads B[l][j] = XT[l][j] = d_l (L^-T)[l][j].
 
+// The same result with the matrix in shared memory (m <= 160), for the sizes the solver runs at:
+// the global-memory version above spends its time in ~3 m barriers around L2 round trips and in
+// a forward substitution that keeps m threads busy.  Here
+//   - the factorisation takes one barrier per column: at step j every thread reads the pivot for
+//     itself, the trailing block is updated with the still unscaled column j (factor 1 / pivot),
+//     and column j is scaled one step later, when nobody reads it any more;
+//   - L is inverted in place from the last column backwards: column j of L^-1 is minus the
+//     already inverted trailing block times column j of L, a row per warp.
+// Rows are padded to an odd stride so that column accesses do not collide in the banks.
+constexpr int kCholSmemRitz = 160;
+__global__ void __launch_bounds__(1024) chol_inv_smem_kernel(const double *S, double *XT, int m, int *dead) {
+    extern __shared__ double chol_dyn[];
+    double *A = chol_dyn;
+    __shared__ double s_dinv[kCholSmemRitz], s_diag[kCholSmemRitz];
+    __shared__ int s_dead0[kCholSmemRitz], s_dead[kCholSmemRitz];
+    const int tid = threadIdx.x, nt = blockDim.x, ty = tid >> 5, tx = tid & 31;
+    const int ld = m + 1;
+    for (int j = tid; j < m; j += nt) {
+        const double p = S[(int64_t)j * m + j];
+        const bool ok = (p > 0.0) && isfinite(p);
+        s_dinv[j] = ok ? 1.0 / sqrt(p) : 0.0;
+        s_dead0[j] = ok ? 0 : 1;
+    }
+    __syncthreads();
+    for (int e = tid; e < m * m; e += nt) {
+        const int i = e / m, j = e % m;
+        A[i * ld + j] = S[e] * s_dinv[i] * s_dinv[j];
+    }
+    __syncthreads();
+    double inv_prev = 0.0;
+    for (int j = 0; j < m; ++j) {
+        const double p = A[j * ld + j];
+        const bool dj = s_dead0[j] || !(p > 1e-10);
+        const double d = dj ? 1.0 : sqrt(p);
+        const double inv = dj ? 0.0 : 1.0 / d;
+        if (tid == 0) { s_dead[j] = dj ? 1 : 0; s_diag[j] = d; }
+        if (j > 0)   // column j - 1 becomes L (zero for a dead column: no coupling to the rest)
+            for (int i = j + tid; i < m; i += nt) A[i * ld + j - 1] = inv_prev == 0.0 ? 0.0 : A[i * ld + j - 1] * inv_prev;
+        if (!dj) {   // trailing update of the lower triangle: A[i][l] -= L[i][j] L[l][j], j < l <= i
+            const double inv2 = inv * inv;
+            for (int i = j + 1 + ty; i < m; i += 32) {
+                const double aij = A[i * ld + j] * inv2;
+                for (int l = j + 1 + tx; l <= i; l += 32) A[i * ld + l] -= aij * A[l * ld + j];
+            }
+        }
+        inv_prev = inv;
+        __syncthreads();
+    }
+    // diagonal of L^-1 into the diagonal of A
+    for (int j = tid; j < m; j += nt) A[j * ld + j] = 1.0 / s_diag[j];
+    __syncthreads();
+    for (int j = m - 2; j >= 0; --j) {
+        const double xjj = A[j * ld + j];
+        double mine[(kCholSmemRitz + 31) / 32];
+        int n = 0;
+        for (int i = j + 1 + ty; i < m; i += 32, ++n) {   // X[i][j] = -x_jj sum_{j < l <= i} X[i][l] L[l][j]
+            double acc = 0.0;
+            for (int l = j + 1 + tx; l <= i; l += 32) acc += A[i * ld + l] * A[l * ld + j];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+            mine[n] = -xjj * acc;
+        }
+        __syncthreads();   // column j of L has been read by everyone
+        n = 0;
+        for (int i = j + 1 + ty; i < m; i += 32, ++n)
+            if (tx == 0) A[i * ld + j] = mine[n];
+        __syncthreads();
+    }
+    // XT[l][j] = d_l X[j][l] for j >= l, zero above; dead output columns are zeroed
+    for (int e = tid; e < m * m; e += nt) {
+        const int l = e / m, j = e % m;
+        XT[e] = (s_dead[j] || j < l) ? 0.0 : A[j * ld + l] * s_dinv[l];
+    }
+    for (int j = tid; j < m; j += nt) dead[j] = s_dead[j];
+}
+
 // fresh pseudo-random entries for the columns marked dead (salted by `salt`)
 __global__ void reseed_dead_kernel(double *Q, int D, int m, const int *dead, uint64_t salt) {
     for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < (int64_t)D * m;
@@ -449,6 +526,60 @@ jacobi_kernel(double *S_g, double *W_g, double *Wout, double *theta, int m, doub
     if (tid == 0 && sweeps_out) *sweeps_out = (double)sweep;
 }
 
+// ---------------------------------------------------------------------------------------
+// Polynomial filter of the subspace iteration (Chebyshev-filtered subspace iteration).
+// With the unwanted part of the spectrum inside [0, b], b = the smallest Ritz value of the block,
+// and c = e = b / 2:
+//   degree 1   Y1 = (G - c) Q / e                 a shifted power step: the k-th wanted direction
+//              gains 2 lambda_k / b - 1 on the unwanted ones, where a plain step gains lambda_k / b;
+//   degree 2   Y2 = T_2((G - c) / e) Q = 2 (G - c) Y1 / e - Q: for the configured power-law spectra
+//              ~10 per two multiplications by G, where two plain steps gain ~2.8.
+// The coefficients come from the Ritz values on the device.  Degree 2 lifts the leading direction
+// over the k-th one by ~(lambda_1 / lambda_k)^2 per iteration; the orthonormalisation that follows
+// works in fp64 and needs the columns to stay independent, so the host asks for it only while
+// that ratio stays below 1e12 (filter_safe_kernel).  When b is not positive against theta_1 (a
+// block wider than the rank of G) the step is a plain power step.
+// ---------------------------------------------------------------------------------------
+struct FilterCoef {
+    double a1, b1, a2, b2, g2;   // Y1 = a1 (G Q) + b1 Q,  Y2 = a2 (G Y1) + b2 Y1 + g2 Q
+    int deg2_safe;
+};
+__device__ __forceinline__ FilterCoef filter_coef(const double *theta, int m, int k) {
+    const double t1 = theta[0], tk = theta[k - 1], b = theta[m - 1];
+    FilterCoef f;
+    const bool shift = isfinite(t1) && isfinite(b) && t1 > 0.0 && b > 1e-12 * t1;
+    if (shift) {
+        const double e = 0.5 * b;
+        const double x1 = (t1 - e) / e, xk = (tk - e) / e;
+        const double g1 = 2.0 * x1 * x1 - 1.0, gk = fabs(2.0 * xk * xk - 1.0);
+        f.deg2_safe = g1 <= 1e12 * fmax(gk, 1.0) ? 1 : 0;
+        f.a1 = 1.0 / e; f.b1 = -1.0;          // (Z - c Q) / e with c = e
+        f.a2 = 2.0 / e; f.b2 = -2.0; f.g2 = -1.0;
+    } else {
+        f.deg2_safe = 0;
+        f.a1 = (isfinite(t1) && t1 > 0.0) ? 1.0 / t1 : 1.0;
+        f.b1 = 0.0;
+        f.a2 = f.a1; f.b2 = 0.0; f.g2 = 0.0;   // (never used: the host takes degree 1 when deg2_safe is 0)
+    }
+    return f;
+}
+__global__ void filter_safe_kernel(const double *theta, int m, int k, double *flag) {
+    *flag = (double)filter_coef(theta, m, k).deg2_safe;
+}
+// Y1 <- a1 Y1 + b1 Q   (Y1 holds G Q on entry)
+__global__ void filter_first_kernel(double *Y1, const double *Q, const double *theta, int m, int k, int64_t n) {
+    const FilterCoef f = filter_coef(theta, m, k);
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x)
+        Y1[e] = f.a1 * Y1[e] + f.b1 * Q[e];
+}
+// Y2 <- a2 Y2 + b2 Y1 + g2 Q   (Y2 holds G Y1 on entry)
+__global__ void filter_second_kernel(double *Y2, const double *Y1, const double *Q, const double *theta, int m, int k,
+                                     int64_t n) {
+    const FilterCoef f = filter_coef(theta, m, k);
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x)
+        Y2[e] = f.a2 * Y2[e] + f.b2 * Y1[e] + f.g2 * Q[e];
+}
+
 // resid[j] = | Z[:, j] - theta[j] Q[:, j] |_2  for j < k;  one CTA per column
 __global__ void residual_kernel(const double *Z, const double *Q, const double *theta, int D, int m,
                                 double *resid) {
@@ -557,7 +688,16 @@ int orthonormalize(double *Zin, double *T, double *S, double *X, int *dead, int 
         int rc = dgemm<double, double, true>(src, m, src, m, S, m, m, m, D, false, false, s, ps);
         if (rc) return rc;
         symmetrize_kernel<<<grid_for((int64_t)m * m), 256, 0, s>>>(S, m, 1);
-        chol_inv_kernel<<<1, 1024, 0, s>>>(S, X, m, dead);
+        if (m <= kCholSmemRitz) {
+            const size_t cb = (size_t)m * (m + 1) * 8;
+            if (cb > 40 * 1024) {   // per call: the attribute belongs to the current device's copy of the kernel
+                rc = record_cuda(cudaFuncSetAttribute(chol_inv_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cb));
+                if (rc) return rc;
+            }
+            chol_inv_smem_kernel<<<1, 1024, cb, s>>>(S, X, m, dead);
+        } else {
+            chol_inv_kernel<<<1, 1024, 0, s>>>(S, X, m, dead);
+        }
         count_launch(2);
         rc = dgemm<double, double, false>(src, m, X, m, dst, m, D, m, m, false, false, s);
         if (rc) return rc;
@@ -621,66 +761,84 @@ int calib_finish(int D, int k, float *Vk, double *lambda, double *trace, double 
         *z = o[0]; *t = o[1];
     };
 
-    // A Ritz iteration: Z = G Q; Rayleigh-Ritz on span(Q) (S = Q^T Z = W Theta W^T, Q <- Q W,
-    // Z <- Z W); residual check; Q <- orthonormalise(Z).  The Ritz rotation keeps the columns
-    // of Z close to mutually orthogonal, which is what the scaled Cholesky-QR relies on.
+    // One iteration: Z = G Q; on a Ritz iteration Rayleigh-Ritz on span(Q) (S = Q^T Z = W Theta W^T,
+    // Q <- Q W, Z <- Z W: no further product with G) and the residual check; then the polynomial
+    // filter on top of Z (degree 2: one more product with G) and Q <- orthonormalise(filtered block).
+    // The Rayleigh-Ritz step (the m x m eigen-problem is the serial, single-CTA part) runs on the
+    // first iterations, which turn the random start block into ordered eigenvector estimates and
+    // give the filter its bounds, and on every second one after that (every fourth with the
+    // degree-1 filter); in between, the QR step takes out of every column its components along the
+    // columns before it, so the columns stay ordered and nearly orthogonal and the scaled
+    // Cholesky-QR stays well conditioned.
     const double tol = 1e-12;
     const int max_mult = 200;
     double max_rel = 1.0;
-    int mult = 0;
+    int mult = 0, degree = 1;
     bool converged = false;
-    while (mult < max_mult) {
+    const int64_t nelem = (int64_t)D * m;
+    for (int iter = 1;; ++iter) {
+        const bool last = mult + 4 > max_mult;   // no room for another whole iteration after this one
         double *Z, *T;
         others(Q, &Z, &T);
         rc = dgemm<double, double, true>(G, D, Q, m, Z, m, D, m, D, false, false, s, ps);   // Z = G Q
         if (rc) return rc;
         ++mult;
-        // The Rayleigh-Ritz step (the m x m eigen-problem is the serial, single-CTA part of an
-        // iteration) runs on the first iterations, which turn the random start block into ordered
-        // eigenvector estimates, and on every fourth one after that; in between the iteration is plain
-        // orthogonal iteration, Q <- orthonormalise(G Q): the QR step takes out of every column its
-        // components along the columns before it, so the columns stay ordered and nearly orthogonal
-        // and the scaled Cholesky-QR stays well conditioned.
-        const bool ritz_step = mult <= 4 || (mult % 4) == 0 || mult == max_mult;
-        if (!ritz_step) {
-            rc = orthonormalize(Z, T, S, X, dead, D, m, (uint64_t)mult + 1, &Q, s, ps);
+        const bool ritz_step = iter <= 3 || (degree == 2 ? (iter & 1) != 0 : (iter % 4) == 0) || last;
+        double *block = Q, *image = Z, *spare = T;   // the filter acts on (block, G block); spare is free
+        if (ritz_step) {
+            rc = dgemm<double, double, true>(Q, m, Z, m, S, m, m, m, D, false, false, s, ps);   // S = Q^T Z
             if (rc) return rc;
-            continue;
-        }
-        rc = dgemm<double, double, true>(Q, m, Z, m, S, m, m, m, D, false, false, s, ps);   // S = Q^T Z
-        if (rc) return rc;
-        symmetrize_kernel<<<grid_for((int64_t)m * m), 256, 0, s>>>(S, m, 1);
-        {
-            const size_t jb = 2 * (size_t)m * m * 8;
-            const bool fits = jb <= kJacobiSmemMax;
-            if (fits && jb > 40 * 1024) {   // per call: the attribute belongs to the current device's copy of the kernel
-                rc = record_cuda(cudaFuncSetAttribute(jacobi_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kJacobiSmemMax));
-                if (rc) return rc;
+            symmetrize_kernel<<<grid_for((int64_t)m * m), 256, 0, s>>>(S, m, 1);
+            {
+                const size_t jb = 2 * (size_t)m * m * 8;
+                const bool fits = jb <= kJacobiSmemMax;
+                if (fits && jb > 40 * 1024) {   // per call: the attribute belongs to the current device's copy of the kernel
+                    rc = record_cuda(cudaFuncSetAttribute(jacobi_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kJacobiSmemMax));
+                    if (rc) return rc;
+                }
+                jacobi_kernel<<<1, kJacobiThreads, fits ? jb : 0, s>>>(S, X, W, theta, m, scal + 2, fits ? 1 : 0);
             }
-            jacobi_kernel<<<1, kJacobiThreads, fits ? jb : 0, s>>>(S, X, W, theta, m, scal + 2, fits ? 1 : 0);
-        }
-        count_launch(2);
-        rc = dgemm<double, double, false>(Q, m, W, m, T, m, D, m, m, false, false, s);  // ritz = Q W
-        if (rc) return rc;
-        rc = dgemm<double, double, false>(Z, m, W, m, Q, m, D, m, m, false, false, s);  // image = Z W
-        if (rc) return rc;
-        double *ritz = T, *image = Q;   // `Z` is free scratch from here on
-        const bool check = (mult >= 4 && (mult % 2) == 0) || mult == max_mult;
-        if (check) {
-            residual_kernel<<<k, 256, 0, s>>>(image, ritz, theta, D, m, resid);
-            max_residual_kernel<<<1, 32, 0, s>>>(resid, theta, k, scal);
             count_launch(2);
-            rc = record_cuda(cudaMemcpyAsync(&max_rel, scal + 1, sizeof(double), cudaMemcpyDeviceToHost, s));
+            rc = dgemm<double, double, false>(Q, m, W, m, T, m, D, m, m, false, false, s);  // ritz = Q W
+            if (rc) return rc;
+            rc = dgemm<double, double, false>(Z, m, W, m, Q, m, D, m, m, false, false, s);  // image = Z W
+            if (rc) return rc;
+            block = T; image = Q; spare = Z;
+            if (iter >= 2) {
+                residual_kernel<<<k, 256, 0, s>>>(image, block, theta, D, m, resid);
+                max_residual_kernel<<<1, 32, 0, s>>>(resid, theta, k, scal);
+                count_launch(2);
+            }
+            filter_safe_kernel<<<1, 1, 0, s>>>(theta, m, k, scal + 3);
+            count_launch();
+            double back[3] = {1.0, 0.0, 0.0};   // scal[1..3]: max relative residual, Jacobi sweeps, degree-2 flag
+            rc = record_cuda(cudaMemcpyAsync(back, scal + 1, sizeof(back), cudaMemcpyDeviceToHost, s));
             if (rc) return rc;
             rc = record_cuda(cudaStreamSynchronize(s));
             if (rc) return rc;
-            if (max_rel <= tol || mult == max_mult) {
-                converged = max_rel <= tol;
-                Q = ritz;
-                break;
+            degree = back[2] != 0.0 ? 2 : 1;
+            if (iter >= 2) {
+                max_rel = back[0];
+                if (max_rel <= tol || last) {
+                    converged = max_rel <= tol;
+                    Q = block;
+                    break;
+                }
             }
         }
-        rc = orthonormalize(image, Z, S, X, dead, D, m, (uint64_t)mult + 1, &Q, s, ps);
+        filter_first_kernel<<<grid_for(nelem), 256, 0, s>>>(image, block, theta, m, k, nelem);           // Y1, in place
+        count_launch();
+        if (degree == 1) {
+            rc = orthonormalize(image, spare, S, X, dead, D, m, (uint64_t)mult + 1, &Q, s, ps);
+            if (rc) return rc;
+            continue;
+        }
+        rc = dgemm<double, double, true>(G, D, image, m, spare, m, D, m, D, false, false, s, ps);       // G Y1
+        if (rc) return rc;
+        ++mult;
+        filter_second_kernel<<<grid_for(nelem), 256, 0, s>>>(spare, image, block, theta, m, k, nelem);  // Y2, in place
+        count_launch();
+        rc = orthonormalize(spare, image, S, X, dead, D, m, (uint64_t)mult + 1, &Q, s, ps);
         if (rc) return rc;
     }
 
