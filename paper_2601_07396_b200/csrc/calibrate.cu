@@ -527,6 +527,155 @@ jacobi_kernel(double *S_g, double *W_g, double *Wout, double *theta, int m, doub
 }
 
 // ---------------------------------------------------------------------------------------
+// The same eigen-decomposition for Ritz matrices whose S and W do not fit in shared memory
+// together (113 < m <= 160, i.e. k = 128): S alone lives in shared memory, and the eigenvector
+// matrix is not touched during the sweeps at all -- every rotation's (c, s) goes to a log in
+// global memory (the pairs of a round follow from its number), and apply_rotations_kernel
+// forms W = J_1 J_2 ... afterwards, a warp per row of W, rows being independent.  With both
+// matrices in global memory a call took 13.6 ms at m = 160, every round a chain of L2 round trips.
+//   head[0] = rounds logged, head[1 + j] = rank of eigenvalue j (descending); log after kJacobiLogHead bytes
+// ---------------------------------------------------------------------------------------
+constexpr int kJacobiLogRitz = 160;
+constexpr size_t kJacobiLogHead = 1024;
+constexpr int kJacobiMaxSweeps = 40;
+
+__device__ __forceinline__ void jacobi_pair(int r, int B, int m, int &p, int &q) {
+    if (B == 0) { p = m - 1; q = r; }
+    else { p = (r + B) % (m - 1); q = (r - B + (m - 1)) % (m - 1); }
+    if (p > q) { const int t = p; p = q; q = t; }
+}
+
+__global__ void __launch_bounds__(1024)
+jacobi_logged_kernel(const double *S_g, double *theta, int m, double *sweeps_out, int *head, double2 *log) {
+    extern __shared__ double jacobi_dyn[];
+    double *S = jacobi_dyn;
+    __shared__ double cs_c[kJacobiLogRitz / 2], cs_s[kJacobiLogRitz / 2];
+    __shared__ int pr_p[kJacobiLogRitz / 2], pr_q[kJacobiLogRitz / 2];
+    __shared__ int s_rot;
+    __shared__ double s_diag[kJacobiLogRitz];
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int h = m / 2;
+    for (int e = tid; e < m * m; e += nt) S[e] = S_g[e];
+    __syncthreads();
+    int sweep = 0, round = 0;
+    for (; sweep < kJacobiMaxSweeps; ++sweep) {
+        if (tid == 0) s_rot = 0;
+        __syncthreads();
+        for (int r = 0; r < m - 1; ++r, ++round) {
+            if (tid < h) {
+                int p, q;
+                jacobi_pair(r, tid, m, p, q);
+                pr_p[tid] = p; pr_q[tid] = q;
+                const double app = S[p * m + p], aqq = S[q * m + q], apq = S[p * m + q];
+                double c = 1.0, sn = 0.0;
+                const double pq2 = apq * apq, dd = fabs(app * aqq);
+                if (apq != 0.0 && pq2 > 1e-34 * dd) {
+                    const double tau = (aqq - app) / (2.0 * apq);
+                    const double t = (tau >= 0.0 ? 1.0 : -1.0) / (fabs(tau) + sqrt(1.0 + tau * tau));
+                    c = rsqrt(1.0 + t * t);
+                    sn = t * c;
+                    if (pq2 > 1e-30 * dd) atomicAdd(&s_rot, 1);
+                }
+                cs_c[tid] = c; cs_s[tid] = sn;
+                log[(size_t)round * h + tid] = make_double2(c, sn);
+            }
+            __syncthreads();
+            // S_AB <- J_A^T S_AB J_B with J = [[c, s], [-s, c]] on the (p, q) plane
+            for (int A = tid >> 5; A < h; A += nt >> 5) {
+                const int p = pr_p[A] * m, q = pr_q[A] * m;
+                const double ca = cs_c[A], sa = cs_s[A];
+                for (int B = tid & 31; B < h; B += 32) {
+                    const int u = pr_p[B], v = pr_q[B];
+                    const double cb = cs_c[B], sb = cs_s[B];
+                    const double spu = S[p + u], spv = S[p + v];
+                    const double squ = S[q + u], sqv = S[q + v];
+                    const double rpu = ca * spu - sa * squ, rpv = ca * spv - sa * sqv;
+                    const double rqu = sa * spu + ca * squ, rqv = sa * spv + ca * sqv;
+                    S[p + u] = cb * rpu - sb * rpv;
+                    S[p + v] = sb * rpu + cb * rpv;
+                    S[q + u] = cb * rqu - sb * rqv;
+                    S[q + v] = sb * rqu + cb * rqv;
+                }
+            }
+            __syncthreads();
+        }
+        if (s_rot == 0) { ++sweep; break; }
+        __syncthreads();
+    }
+    // order by descending eigenvalue (rank sort; ties by index)
+    for (int i = tid; i < m; i += nt) s_diag[i] = S[i * m + i];
+    __syncthreads();
+    for (int j = tid; j < m; j += nt) {
+        int rk = 0;
+        const double x = s_diag[j];
+        for (int i = 0; i < m; ++i) rk += (s_diag[i] > x) || (s_diag[i] == x && i < j);
+        head[1 + j] = rk;
+        theta[rk] = x;
+    }
+    if (tid == 0) {
+        head[0] = round;
+        if (sweeps_out) *sweeps_out = (double)sweep;
+    }
+}
+
+// W = product of the logged rotations, columns permuted to descending eigenvalue order.  A warp owns
+// a row of W (initially a unit vector) in shared memory and applies the rounds in order -- the
+// rotations of one round touch disjoint column pairs, one or more per lane; the (c, s) of eight
+// rounds at a time are staged in shared memory for the CTA's eight rows, the next chunk's loads in
+// flight while the current one is applied.
+constexpr int kApplyWarps = 8, kApplyChunk = 8;
+__global__ void __launch_bounds__(kApplyWarps * 32)
+apply_rotations_kernel(const int *head, const double2 *log, double *Wout, int m) {
+    __shared__ double rows[kApplyWarps][kJacobiLogRitz];
+    __shared__ double2 cs[2][kApplyChunk][kJacobiLogRitz / 2];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, h = m / 2;
+    const int row = blockIdx.x * kApplyWarps + warp;
+    for (int j = lane; j < m; j += 32) rows[warp][j] = (j == row) ? 1.0 : 0.0;
+    const int nrounds = head[0];
+    const int nchunks = (nrounds + kApplyChunk - 1) / kApplyChunk;
+    constexpr int kPre = (kApplyChunk * (kJacobiLogRitz / 2) + kApplyWarps * 32 - 1) / (kApplyWarps * 32);
+    double2 pre[kPre];
+    auto fetch = [&](int ch) {
+#pragma unroll
+        for (int i = 0; i < kPre; ++i) {
+            const int e = tid + i * kApplyWarps * 32;
+            const int R = ch * kApplyChunk + e / h;
+            pre[i] = (e < kApplyChunk * h && R < nrounds) ? log[(size_t)R * h + e % h] : make_double2(1.0, 0.0);
+        }
+    };
+    auto stash = [&](int buf) {
+#pragma unroll
+        for (int i = 0; i < kPre; ++i) {
+            const int e = tid + i * kApplyWarps * 32;
+            if (e < kApplyChunk * h) cs[buf][e / h][e % h] = pre[i];
+        }
+    };
+    if (nchunks > 0) { fetch(0); stash(0); }
+    __syncthreads();
+    int r = 0;   // round within its sweep
+    for (int ch = 0; ch < nchunks; ++ch) {
+        if (ch + 1 < nchunks) fetch(ch + 1);
+        double *w = rows[warp];
+        for (int t = 0; t < kApplyChunk && ch * kApplyChunk + t < nrounds; ++t) {
+            for (int B = lane; B < h; B += 32) {
+                int u, v;
+                jacobi_pair(r, B, m, u, v);
+                const double2 f = cs[ch & 1][t][B];
+                const double wu = w[u], wv = w[v];
+                w[u] = f.x * wu - f.y * wv;
+                w[v] = f.y * wu + f.x * wv;
+            }
+            __syncwarp();
+            r = (r + 1 == m - 1) ? 0 : r + 1;
+        }
+        if (ch + 1 < nchunks) stash((ch + 1) & 1);
+        __syncthreads();
+    }
+    if (row < m)
+        for (int j = lane; j < m; j += 32) Wout[(int64_t)row * m + head[1 + j]] = rows[warp][j];
+}
+
+// ---------------------------------------------------------------------------------------
 // Polynomial filter of the subspace iteration (Chebyshev-filtered subspace iteration).
 // With the unwanted part of the spectrum inside [0, b], b = the smallest Ritz value of the block,
 // and c = e = b / 2:
@@ -792,11 +941,26 @@ int calib_finish(int D, int k, float *Vk, double *lambda, double *trace, double 
             {
                 const size_t jb = 2 * (size_t)m * m * 8;
                 const bool fits = jb <= kJacobiSmemMax;
-                if (fits && jb > 40 * 1024) {   // per call: the attribute belongs to the current device's copy of the kernel
-                    rc = record_cuda(cudaFuncSetAttribute(jacobi_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kJacobiSmemMax));
-                    if (rc) return rc;
+                // the rotation log borrows the split products' scratch, which is idle during the Ritz step
+                const size_t log_bytes = kJacobiLogHead + (size_t)kJacobiMaxSweeps * (m - 1) * (m / 2) * sizeof(double2);
+                if (m <= kJacobiLogRitz && ps.buf != nullptr && log_bytes <= ps.bytes) {
+                    const size_t sb = (size_t)m * m * 8;
+                    if (sb > 40 * 1024) {   // per call: the attribute belongs to the current device's copy of the kernel
+                        rc = record_cuda(cudaFuncSetAttribute(jacobi_logged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sb));
+                        if (rc) return rc;
+                    }
+                    int *head = (int *)ps.buf;
+                    double2 *rot = (double2 *)((char *)ps.buf + kJacobiLogHead);
+                    jacobi_logged_kernel<<<1, kJacobiThreads, sb, s>>>(S, theta, m, scal + 2, head, rot);
+                    apply_rotations_kernel<<<(m + kApplyWarps - 1) / kApplyWarps, kApplyWarps * 32, 0, s>>>(head, rot, W, m);
+                    count_launch();
+                } else {
+                    if (fits && jb > 40 * 1024) {   // per call: the attribute belongs to the current device's copy of the kernel
+                        rc = record_cuda(cudaFuncSetAttribute(jacobi_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kJacobiSmemMax));
+                        if (rc) return rc;
+                    }
+                    jacobi_kernel<<<1, kJacobiThreads, fits ? jb : 0, s>>>(S, X, W, theta, m, scal + 2, fits ? 1 : 0);
                 }
-                jacobi_kernel<<<1, kJacobiThreads, fits ? jb : 0, s>>>(S, X, W, theta, m, scal + 2, fits ? 1 : 0);
             }
             count_launch(2);
             rc = dgemm<double, double, false>(Q, m, W, m, T, m, D, m, m, false, false, s);  // ritz = Q W
