@@ -40,7 +40,7 @@ NOMINAL_HBM_GBS = 8000.0
 # summaries under profiles/ name the commands).  Keyed by (workload, blocks, kernel family);
 # any other shape reports null -- nothing is scaled.
 NCU_TRAFFIC_BYTES = {
-    "cached": {("flux", 57, 2): 3270419968},   # profiles/umma_cached_kernel_flux_57blocks_traffic.txt
+    "cached": {("flux", 57, 2): 3269659648},   # profiles/umma_cached_kernel_flux_57blocks_traffic.txt
     "full": {("flux", 57, 2): 4303533312},     # profiles/umma_full_kernel_flux_57blocks_traffic.txt
 }
 
