@@ -652,21 +652,34 @@ apply_rotations_kernel(const int *head, const double2 *log, double *Wout, int m)
     };
     if (nchunks > 0) { fetch(0); stash(0); }
     __syncthreads();
-    int r = 0;   // round within its sweep
+    // the pairs of this lane's B = lane, lane + 32, ...: p = (r + B) mod (m - 1) and q = (r - B) mod (m - 1)
+    // both step up by one from a round to the next (pair 0 keeps p = m - 1), so no round needs a division
+    constexpr int kPairs = (kJacobiLogRitz / 2 + 31) / 32;
+    int pp[kPairs], qq[kPairs];
+#pragma unroll
+    for (int i = 0; i < kPairs; ++i) {
+        const int B = lane + 32 * i;
+        pp[i] = B == 0 ? m - 1 : B % (m - 1);
+        qq[i] = B == 0 ? 0 : (m - 1 - B % (m - 1)) % (m - 1);
+    }
     for (int ch = 0; ch < nchunks; ++ch) {
         if (ch + 1 < nchunks) fetch(ch + 1);
         double *w = rows[warp];
         for (int t = 0; t < kApplyChunk && ch * kApplyChunk + t < nrounds; ++t) {
-            for (int B = lane; B < h; B += 32) {
-                int u, v;
-                jacobi_pair(r, B, m, u, v);
-                const double2 f = cs[ch & 1][t][B];
-                const double wu = w[u], wv = w[v];
-                w[u] = f.x * wu - f.y * wv;
-                w[v] = f.y * wu + f.x * wv;
+#pragma unroll
+            for (int i = 0; i < kPairs; ++i) {
+                const int B = lane + 32 * i;
+                if (B < h) {
+                    const int u = min(pp[i], qq[i]), v = max(pp[i], qq[i]);
+                    const double2 f = cs[ch & 1][t][B];
+                    const double wu = w[u], wv = w[v];
+                    w[u] = f.x * wu - f.y * wv;
+                    w[v] = f.y * wu + f.x * wv;
+                }
+                if (B != 0) pp[i] = pp[i] + 1 == m - 1 ? 0 : pp[i] + 1;
+                qq[i] = qq[i] + 1 == m - 1 ? 0 : qq[i] + 1;
             }
             __syncwarp();
-            r = (r + 1 == m - 1) ? 0 : r + 1;
         }
         if (ch + 1 < nchunks) stash((ch + 1) & 1);
         __syncthreads();
