@@ -52,6 +52,7 @@ struct UmmaParams {
     float beta;
     float beta_r;          // full step: EMA weight of the stored residual (0: the residual is replaced)
     size_t r_off;          // offset of R in a block's state
+    int r_slots;           // full step with residual EMA: slots of the ring the old R streams through
 };
 
 struct SmemLayout {
@@ -666,14 +667,19 @@ template <bool kTmemA, bool kResEma>
 __global__ void __launch_bounds__(kThreadsFull, 1)
 umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant__ CUtensorMap tm_vt,
                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_rout,
-                 const __grid_constant__ CUtensorMap tm_chat, const UmmaParams p) {
+                 const __grid_constant__ CUtensorMap tm_chat, const __grid_constant__ CUtensorMap tm_rold,
+                 const UmmaParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t a_base = base;                                     // A operand (and, for k >= 64, staged Chat)
     const uint32_t chat_base = a_base + p.chat_stage_off;             // == a_base when k >= 64
     const uint32_t v_base0 = a_base + p.a_region_bytes;
     const uint32_t stage0 = v_base0 + (uint32_t)p.v_slots * p.vslice_bytes;
-    const Bars bar = bars_at(stage0 + (uint32_t)p.stages * kTileBytes);
+    // residual EMA (kResEma): the stored R streams through r_slots slots after the F ring, whose
+    // barriers are entries stages .. stages + r_slots - 1 of the ring's barrier arrays
+    const uint32_t rold0 = stage0 + (uint32_t)p.stages * kTileBytes;
+    const int r_slots = kResEma ? p.r_slots : 0;
+    const Bars bar = bars_at(rold0 + (uint32_t)r_slots * kTileBytes);
     // barriers beyond the ring ones: c_full (C accumulated), a_full (A operand written),
     // p2_done (pass-2 MMAs of the unit finished: the A region may be restaged), chat_full
     // (previous Chat staged)
@@ -699,6 +705,8 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
         // F slot: free again after five arrivals -- pass 1: the MMAs' commit plus four from the
         // MMA thread; pass 2: the four slab stores plus the MMA thread's "seen" (see there)
         for (int s = 0; s < p.stages; ++s) { mbar_init(bar.full + 8 * s, 1); mbar_init(bar.empty + 8 * s, 5); }
+        // old-R slot: free again once the four warps of the chunk's epilogue group have read it
+        for (int s = p.stages; s < p.stages + r_slots; ++s) { mbar_init(bar.full + 8 * s, 1); mbar_init(bar.empty + 8 * s, 4); }
         for (int s = 0; s < p.acc_stages; ++s) { mbar_init(bar.acc_full + 8 * s, 1); mbar_init(bar.acc_empty + 8 * s, 8); }
         for (int s = 0; s < p.v_slots; ++s) { mbar_init(bar.v_full + 8 * s, 1); mbar_init(bar.v_empty + 8 * s, 1); }
         mbar_init(bar.a_full, c_split ? 256 : 128);
@@ -712,6 +720,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
         prefetch_tensormap(&tm_v);
         prefetch_tensormap(&tm_rout);
         prefetch_tensormap(&tm_chat);
+        if constexpr (kResEma) prefetch_tensormap(&tm_rold);
     }
     if (warp == 1) {
         tmem_alloc(bar.tmem_slot, tmem_cols);
@@ -750,6 +759,33 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                             if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; }
                         }
                     }
+            }
+        }
+        if constexpr (kResEma) {
+            // Third request stream (residual EMA of the ablation, Sec. 4.5): the chunks of the stored R,
+            // in the order pass 2 meets them.  A block's first full step blends nothing and asks for none.
+            if (lane == 1) {
+                RingPos rr;
+                uint32_t ir = 0;
+                for (int u = cid; u < p.units; u += nctas) {
+                    const Unit un = decode_unit(p, u);
+                    if (*(volatile uint32_t *)&header_of(p, un.b)->full_steps == 0) continue;
+                    for (int g = 0; g < G; ++g) {
+                        const int cg = (G - 1 - g) * p.gc;
+                        const int nsub = min(p.gc, CT - cg);
+                        for (int j = 0; j < nsub; ++j, ++ir) {
+                            const uint32_t sl = (uint32_t)p.stages + rr.idx;
+                            if (!mbar_wait(bar.empty + 8 * sl, rr.ph ^ 1u, abort_flag, 102)) {
+                                record_timeout(p, abort_flag, ir, (uint32_t)g);
+                                goto done;
+                            }
+                            mbar_arrive_expect_tx(bar.full + 8 * sl, kTileBytes);
+                            tma_load_3d(rold0 + rr.idx * kTileBytes, &tm_rold, bar.full + 8 * sl, (cg + j) * kTileCols,
+                                        un.rt * kTileRows, un.b);
+                            rr.step((uint32_t)r_slots);
+                        }
+                    }
+                }
             }
         }
     } else if (warp == kFullVWarp) {
@@ -876,7 +912,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
         const uint32_t chat_row_bytes = p.k >= 32 ? 128u : (uint32_t)p.k * 4u;
         const int nblk = (p.k + 31) / 32;
         uint32_t it = 0, ig = 0, ui = 0, nchat = 0;   // F chunks, pass-2 groups, units, Chat tiles consumed
-        RingPos fr, ar;                               // ring positions of chunk `it`, group `ig`
+        RingPos fr, ar, ro;                           // ring positions of chunk `it`, group `ig`, old-R chunk
         int prev_slot = -1;                           // slot whose slab store may still be reading
         const bool defer_release = p.stages >= 4;
         // R is not read again by this step: its lines are the first to go, which leaves more of L2 to
@@ -1081,6 +1117,7 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
             }
             // ---- epilogue duty for this group's chunks of pass 2
             const bool first_unit = kResEma && *(volatile uint32_t *)&header_of(p, un.b)->full_steps == 0;
+            const bool blend = kResEma && !first_unit;   // every pass-2 chunk of this unit has an old-R chunk in the ring
             const int slab_row0 = un.rt * kTileRows + q * kSlabRows;
             const bool slab_live = (int64_t)slab_row0 < p.N;
             it += CT;   // pass-1 slots are consumed by the MMA warp alone
@@ -1095,23 +1132,22 @@ umma_full_kernel(const __grid_constant__ CUtensorMap tm_f, const __grid_constant
                 if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar.acc_full + 8 * as, aph, abort_flag, 16))) { record_timeout(p, abort_flag, it, ig, ui); goto done; }
                 SVDC_TRACE_ADD(3, e3);
                 if (last_own < 0 && lane == 0) mbar_arrive(bar.acc_empty + 8 * as);
-                for (int j = 0; j < nsub; ++j, ++it, fr.step((uint32_t)p.stages)) {
+                for (int j = 0; j < nsub; ++j, ++it, fr.step((uint32_t)p.stages), (blend ? ro.step((uint32_t)r_slots) : (void)0)) {
                     if ((it & 1u) != grp) continue;
                     const int c = cg + j;
                     const uint32_t s = fr.idx, ph = fr.ph;
-                    // residual EMA (ablation): this row's 64 columns of the stored R, asked for before the
-                    // waits below so that the loads are under way while the chunk and its accumulator arrive
+                    // residual EMA (ablation): this row's 64 columns of the stored R, from the old-R ring (rows
+                    // past N and columns past D arrive as zeros and are never stored)
                     uint4 r_old[kResEma ? 8 : 1];
-                    bool blend = false;
                     if constexpr (kResEma) {
-                        const int64_t n = (int64_t)un.rt * kTileRows + row;
-                        blend = !first_unit && n < p.N;
                         if (blend) {
-                            const uint4 *src = reinterpret_cast<const uint4 *>(p.state + (size_t)un.b * p.state_stride + p.r_off +
-                                                                               ((size_t)n * p.D + (size_t)c * kTileCols) * 2);
+                            const uint32_t sl = (uint32_t)p.stages + ro.idx;
+                            if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar.full + 8 * sl, ro.ph, abort_flag, 20))) { record_timeout(p, abort_flag, it, ig, ui); goto done; }
+                            const uint32_t otile = rold0 + ro.idx * kTileBytes + (uint32_t)row * 128u;
 #pragma unroll
-                            for (int cc = 0; cc < 8; ++cc)
-                                r_old[cc] = (c * kTileCols + cc * 8 < p.D) ? __ldcg(src + cc) : make_uint4(0u, 0u, 0u, 0u);
+                            for (int cc = 0; cc < 8; ++cc) r_old[cc] = lds128(otile + (((uint32_t)cc) ^ ((uint32_t)row & 7u)) * 16u);
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(bar.empty + 8 * sl);
                         }
                     }
                     SVDC_TRACE_MARK(e4);
@@ -1341,10 +1377,22 @@ bool fill_full(const StepArgs &a, UmmaParams &p) {
     p.stages = stages_for(p.v_slots);
     if (p.stages < 2) return false;
     p.a_bufs = 1;
+    p.r_slots = 0;
+    if (a.beta_r > 0.0f) {
+        // residual EMA: the old R is a third stream, as many bytes as F -- it takes up to four slots,
+        // from the F ring (down to six slots) and, before that, from the basis ring (down to two)
+        auto room = [&]() { return (int)((avail - (size_t)p.a_region_bytes - (size_t)p.v_slots * p.vslice_bytes) / kTileBytes); };
+        while (p.v_slots > 2 && room() < 6 + 4) --p.v_slots;
+        const int slots = room() < kMaxStages ? room() : kMaxStages;
+        p.r_slots = slots - 6 < 4 ? slots - 6 : 4;
+        if (p.r_slots < 2) { p.r_slots = 2; }
+        p.stages = (slots - p.r_slots) & ~1;
+        if (p.stages < 2) return false;
+    }
     return true;
 }
 size_t smem_bytes_full(const UmmaParams &p) {
-    return 1024 + (size_t)p.a_region_bytes + (size_t)p.v_slots * p.vslice_bytes + (size_t)p.stages * kTileBytes +
+    return 1024 + (size_t)p.a_region_bytes + (size_t)p.v_slots * p.vslice_bytes + (size_t)(p.stages + p.r_slots) * kTileBytes +
            kBarBytes + 64;
 }
 
@@ -1512,7 +1560,7 @@ int umma_full_step(const StepArgs &a, cudaStream_t s) {
 
     const StateLayout SL = state_layout(a.N, a.D, a.k, a.dtype);
     const BasisLayout BL = basis_layout(a.D, a.k, a.dtype);
-    CUtensorMap tm_f, tm_vt, tm_v, tm_rout, tm_chat;
+    CUtensorMap tm_f, tm_vt, tm_v, tm_rout, tm_chat, tm_rold;
     int rc = make_map(&tm_f, a.F, a.D, a.N, a.nblocks, (uint64_t)a.ld * 2, a.F_stride, kTileCols, kTileRows);
     if (rc) return rc;
     rc = make_map(&tm_vt, (const char *)a.basis + BL.vt_bf16, a.D, a.k, a.nblocks, (uint64_t)a.D * 2,
@@ -1527,6 +1575,10 @@ int umma_full_step(const StepArgs &a, cudaStream_t s) {
     rc = make_map(&tm_chat, (char *)a.state + SL.chat, a.k, a.N, a.nblocks, (uint64_t)a.k * 4, a.state_stride,
                   a.k < 32 ? a.k : 32, kTileRows, 4);
     if (rc) return rc;
+    // the stored R as whole chunks, for the residual EMA's third stream (unused otherwise)
+    rc = make_map(&tm_rold, (const char *)a.state + SL.r, a.D, a.N, a.nblocks, (uint64_t)a.D * 2, a.state_stride,
+                  kTileCols, kTileRows);
+    if (rc) return rc;
 
     const size_t smem = smem_bytes_full(p);
     const int sms = num_sms();
@@ -1534,11 +1586,11 @@ int umma_full_step(const StepArgs &a, cudaStream_t s) {
     auto launch = [&](auto kern) {
         const int rc_attr = allow_big_smem(kern, kSmemBudget);
         if (rc_attr) return rc_attr;
-        kern<<<grid, kThreadsFull, smem, s>>>(tm_f, tm_vt, tm_v, tm_rout, tm_chat, p);
+        kern<<<grid, kThreadsFull, smem, s>>>(tm_f, tm_vt, tm_v, tm_rout, tm_chat, tm_rold, p);
         return (int)SVDCACHE_OK;
     };
     // operand in tensor memory from k = 64 on (fill_full has sized the rings for it); the residual EMA
-    // of the ablation is an instantiation of its own (its old-R loads cost registers)
+    // of the ablation is an instantiation of its own (a third TMA stream and ring for the old R)
     const bool ema = a.beta_r > 0.0f;
     if (a.k >= 64) rc = ema ? launch(umma_full_kernel<true, true>) : launch(umma_full_kernel<true, false>);
     else rc = ema ? launch(umma_full_kernel<false, true>) : launch(umma_full_kernel<false, false>);

@@ -168,6 +168,35 @@ def test_residual_ema_full_step(N, D, k, dtype):
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("k", [64, 128])
+def test_residual_ema_batch_with_blocks_at_their_first_step(k):
+    """One batched launch in which some blocks blend with a stored residual and others are at their
+    first full step (nothing to blend, nothing fetched): bitwise the per-block calls.  Enough row
+    tiles that every CTA meets both kinds, in either order."""
+    N, D, dt, nb = 5000, 1024, sc.BF16, 5
+    spec = streams.StreamSpec("ablmix", blocks=nb, rows=N, D=D, dtype="bf16", k=k, T=3, interval=1,
+                              rank=2 * k, amp=30.0, power=1.0, noise_std=0.05)
+    st = [streams.BlockStream(spec, b, device=DEV) for b in range(nb)]
+    bases = torch.stack([sc.svdcache_basis_prepare(st[b].V_gen[:, :k].float().contiguous(), dt) for b in range(nb)])
+    s_b = sc.new_state(N, D, k, dt, DEV, blocks=nb)
+    s_s = sc.new_state(N, D, k, dt, DEV, blocks=nb)
+    seasoned = (0, 2, 3)
+    for b in seasoned:   # these blocks have a stored residual before the batched call
+        for s_ in (s_b, s_s):
+            sc.svdcache_full_step_residual_ema_batched(st[b].features(0), bases[b], s_[b], k, 0.9, 0.5)
+    for t in (1, 2):
+        F = torch.stack([st[b].features(t) for b in range(nb)])
+        sc.svdcache_full_step_residual_ema_batched(F, bases, s_b, k, 0.9, 0.5)
+        for b in range(nb):
+            sc.svdcache_full_step_residual_ema_batched(F[b], bases[b], s_s[b], k, 0.9, 0.5)
+        torch.cuda.synchronize()
+        for b in range(nb):
+            for x, y in zip(sc.state_views(s_b[b], N, D, k, dt), sc.state_views(s_s[b], N, D, k, dt)):
+                assert torch.equal(x, y)
+            assert sc.svdcache_state_query(s_b[b]) == ((t + 1) if b in seasoned else t, 0)
+
+
+@pytest.mark.gpu
 def test_blocks_of_different_rank_in_one_call():
     """Ranks picked per block from its own spectrum (Eq. 6 at tau = 0.85, rounded up to what the
     kernels take), one ranked call over all blocks against per-block calls (bitwise) and the oracle."""
