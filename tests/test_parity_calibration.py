@@ -196,6 +196,22 @@ def test_noise_free_stack_recovers_the_generator_basis():
     assert float(lam.sum()) == pytest.approx(float(tr[0]), rel=1e-6)   # all the energy is in rank 16
 
 
+def test_steep_spectrum_takes_the_one_product_iteration():
+    """A stack whose k-th eigenvalue lies 7 decades under the first: the degree-2 filter would lift
+    the leading direction 1e14 over the k-th one per iteration, so the solver has to fall back to
+    shifted power steps (one product with G per iteration) -- same subspace, same eigenvalues."""
+    M, D, k, r = 3000, 1152, 32, 64
+    g = torch.Generator(device="cpu").manual_seed(1234)
+    A = torch.linalg.qr(torch.randn(M, r, generator=g, dtype=torch.float64))[0]
+    B = torch.linalg.qr(torch.randn(D, r, generator=g, dtype=torch.float64))[0]
+    sv = 10.0 ** (-0.12 * torch.arange(r, dtype=torch.float64))
+    stack = ((A * sv) @ B.t() * 50.0).float().to(DEV)
+    Vk, lam, tr, info = sc.svdcache_calibrate(stack, k)
+    assert info[1] <= 1e-12
+    assert float(lam[0] / lam[k - 1]) > 1e7
+    _compare(stack, k, Vk, lam, tr)
+
+
 def test_rank_selection_by_energy_threshold():
     """Eq. 6 on the calibrated spectrum, against the oracle's rule."""
     spec = streams.TINY
