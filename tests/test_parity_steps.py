@@ -125,6 +125,28 @@ def test_shapes_and_ragged_tails(N, D, k, dtype, ld_pad):
     _play(spec, 0, Vk, range(5), ld_pad=ld_pad)
 
 
+def _random_shapes(n, seed=20260131):
+    """Seeded draw of bf16 shapes the tensor-core kernels take: every rank class (operand in shared
+    memory, in tensor memory with two buffers or one), widths that are not a multiple of the group
+    width, row counts with ragged last tiles, padded leading dimensions."""
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        k = int(rng.choice([16, 32, 64, 128, 192, 256]))
+        D = int(rng.integers(max(k, 64) // 8, 2600 // 8)) * 8
+        N = int(rng.integers(1, 1500))
+        ld_pad = int(rng.choice([0, 8, 64]))
+        out.append((N, D, k, ld_pad))
+    return out
+
+
+@pytest.mark.parametrize("N,D,k,ld_pad", _random_shapes(18))
+def test_random_bf16_shapes(N, D, k, ld_pad):
+    spec = streams.StreamSpec("rand", blocks=1, rows=N, D=D, dtype="bf16", k=k, T=4, interval=2,
+                              rank=min(D, 2 * k), amp=30.0, power=1.0, noise_std=0.02)
+    _play(spec, 0, None, range(4), ld_pad=ld_pad)
+
+
 @pytest.mark.parametrize("D", [256, 448, 704])
 def test_first_full_step_never_reads_the_old_state(D):
     """Narrow blocks with many row tiles: a tile takes fewer chunks than the load ring has slots,
