@@ -205,7 +205,10 @@ def measure_steps(sc, spec, wl, steps, warmup, barrier, sampler=None):
     barrier()
     if sampler is not None:
         sampler.start()
-        time.sleep(0.25)
+        t_wait = time.time()
+        while not sampler.rows and time.time() - t_wait < 3.0:   # nvidia-smi can take a second to print its first line
+            time.sleep(0.02)
+        time.sleep(0.05)
     launches0 = sc.svdcache_kernel_launches()
     events = []
     t_host0 = time.time()
